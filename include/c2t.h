@@ -1,0 +1,254 @@
+/*
+ * libc2t — draft-tree construction for speculative decoding with a confidence
+ * classifier (C2T, arXiv 2502.13652), as CUDA kernels for sm_100a behind a C ABI.
+ *
+ * One context serves B independent sequences on one GPU.  A decode step is
+ *
+ *   c2t_begin_step
+ *   for level = 0 .. D-1:   c2t_expand_level(level, draft logits)   (Sec. 4.2.1, Eq. 1-3)
+ *                           c2t_prune(level)                        (Eq. 4, Alg. 1, Sec. 4.2.2)
+ *                           [caller runs its draft model on the emitted frontier]
+ *   c2t_prune(C2T_FINAL)                                            (Top-N rerank, Sec. 2.2)
+ *   c2t_build_verify                                                (tree attention, Sec. 2.2)
+ *   c2t_accept(target logits)                                       (accept length, Sec. 5 Metrics)
+ *
+ * Conventions, unless a function says otherwise:
+ *   - pointers named *_dev are device pointers, *_host host pointers; "stream" is a
+ *     cudaStream_t passed as void* (NULL = the legacy default stream);
+ *   - every call returns C2T_OK (0) or a negative C2T_E* code; nothing throws, exits
+ *     or prints;
+ *   - calls only enqueue work on `stream` and return; outputs are valid in stream
+ *     order.  Only c2t_status and c2t_decode_step_host synchronise;
+ *   - the library never allocates or frees device memory: the workspace, every input
+ *     and every output belong to the caller, who keeps them alive until the work
+ *     that uses them has finished;
+ *   - a context is not thread-safe; use one context per stream;
+ *   - data faults (NaN or +inf in a logits row, a row of only -inf, a tree that
+ *     outgrows its capacity) never fault the device: they set bits in a per-sequence
+ *     status word and leave that sequence's results unspecified but in bounds.
+ */
+#ifndef C2T_H
+#define C2T_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct c2t_ctx c2t_ctx;
+
+typedef enum { C2T_F32 = 0, C2T_BF16 = 1 } c2t_dtype;
+/* C2T_CLS_MLP: the paper's two-layer FFN.  C2T_CLS_IDENTITY_JOINT: confidence := joint
+ * probability, which turns the method into EAGLE-2's expand + rerank (Sec. 2.2). */
+typedef enum { C2T_CLS_MLP = 0, C2T_CLS_IDENTITY_JOINT = 1 } c2t_classifier;
+/* What "extend N or topK(N) to T" (Alg. 1) adds to the tree at a level: only the capped
+ * next-layer generators, or every node that passed the threshold. */
+typedef enum { C2T_ADD_FRONTIER = 0, C2T_ADD_ALL_SURVIVORS = 1 } c2t_tree_add;
+
+#define C2T_FINAL (-1)
+
+#define C2T_OK       0
+#define C2T_EINVAL  (-1)   /* null pointer, non-positive size, unknown enum value        */
+#define C2T_EALIGN  (-2)   /* logits base or stride not 16-byte aligned                  */
+#define C2T_ERANGE  (-3)   /* a size exceeds a C2T_MAX_* limit or the workspace is small */
+#define C2T_EORDER  (-4)   /* calls out of sequence within a decode step                 */
+#define C2T_ECUDA   (-5)   /* a CUDA runtime call failed                                 */
+
+#define C2T_MAX_BATCH     4096
+#define C2T_MAX_TOPK      32
+#define C2T_MAX_FRONTIER  32
+#define C2T_MAX_HIDDEN    64
+#define C2T_MAX_DEPTH     32
+#define C2T_MAX_BUDGET    1024
+#define C2T_MAX_TREE      8192   /* nodes per sequence before the Top-N rerank */
+
+/* per-sequence status bits */
+#define C2T_ST_NAN_LOGIT     1u
+#define C2T_ST_POSINF_LOGIT  2u
+#define C2T_ST_ALL_NEGINF    4u
+#define C2T_ST_TREE_OVERFLOW 8u
+
+/*
+ * Method parameters (Alg. 1's inputs d_max and beta; Top-K of Sec. 4.2.2 split into the
+ * K children classified per node and the F generators kept per layer, K = F in the
+ * paper; EAGLE-2's N of Sec. 2.2; the classifier of Sec. 4.1).
+ */
+typedef struct {
+  int32_t batch;          /* B sequences                                                  */
+  int32_t vocab;          /* V                                                            */
+  int32_t dtype;          /* c2t_dtype of draft and target logits                         */
+  int32_t max_depth;      /* D = d_max draft rounds                                       */
+  int32_t topk;           /* K                                                            */
+  int32_t frontier_cap;   /* F                                                            */
+  int32_t budget;         /* N, counts the root; 0 = no rerank                            */
+  float   threshold;      /* beta; a node is kept iff C >= beta                           */
+  int32_t entropy_top_m;  /* M of Eq. 3; only 0 (exact entropy, Eq. 2) is implemented     */
+  int32_t classifier;     /* c2t_classifier                                               */
+  int32_t hidden;         /* h                                                            */
+  const float *w1;        /* HOST [h*3] row-major, features in the order (P, H, d)        */
+  const float *b1;        /* HOST [h]                                                     */
+  const float *w2;        /* HOST [h]                                                     */
+  const float *b2;        /* HOST [1]     (all four copied at init; unused in identity mode) */
+  int32_t tree_add;       /* c2t_tree_add                                                 */
+  int32_t device;         /* CUDA device ordinal                                          */
+} c2t_config;
+
+/* Sizes derived from a configuration (0 on an invalid configuration). */
+size_t  c2t_workspace_bytes(const c2t_config *cfg);  /* device workspace the caller provides   */
+int32_t c2t_tree_capacity(const c2t_config *cfg);    /* nodes per sequence before the rerank   */
+int32_t c2t_final_width(const c2t_config *cfg);      /* Nw: node slots per sequence after it   */
+int32_t c2t_mask_words(const c2t_config *cfg);       /* W = ceil(Nw / 64)                      */
+
+/*
+ * Validates cfg, copies the classifier weights to the device and carves `workspace_dev`
+ * (256-byte aligned, at least c2t_workspace_bytes(cfg), owned by the caller for the life
+ * of the context).  Synchronous.  On success *out receives the context.
+ */
+int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes, c2t_ctx **out);
+void c2t_destroy(c2t_ctx *ctx);
+
+/*
+ * Starts a decode step: tree = {root}, C_root = 1, frontier = {root}  (Alg. 1, initialisation).
+ * root_tok_dev [B] int32: the token the target model produced last; prefix_len_dev [B] int32:
+ * tokens already committed (only used for position ids).  Clears the status words.
+ */
+int c2t_begin_step(c2t_ctx *ctx, const int32_t *root_tok_dev, const int32_t *prefix_len_dev,
+                   void *stream);
+
+/*
+ * Post-processing of one draft round (Sec. 4.2.1; Eq. 2; Top-K purpose 1 of Sec. 4.2.2):
+ * for every active frontier slot (b, j), j < n_level(b), one pass over logits row (b, j)
+ * yields the softmax normaliser, the exact entropy of the row and its K most probable
+ * tokens (ties to the lower token id).  Results stay in the workspace for c2t_prune.
+ *   logits_dev: [B, F, V] of cfg.dtype; element offset of (b, j, v) =
+ *               b*seq_stride + j*row_stride + v.  Base address 16-byte aligned, both strides
+ *               multiples of 16 bytes.  Rows of inactive slots are never read.
+ *   level:      must equal the number of c2t_prune calls made since c2t_begin_step.
+ */
+int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t seq_stride,
+                     int64_t row_stride, void *stream);
+
+/* Next-layer generators, written by c2t_prune(level >= 0).  Caller-owned device arrays;
+ * any pointer may be NULL to skip that output. */
+typedef struct {
+  int32_t *count;        /* [B]     n_{level+1}(b) <= F                                   */
+  int32_t *token;        /* [B, F]  token of generator slot j (input of the draft model)  */
+  int32_t *node_id;      /* [B, F]  its id in the tree                                    */
+  int32_t *parent_slot;  /* [B, F]  slot of its parent in the current level's frontier    */
+} c2t_frontier;
+
+/*
+ * level >= 0 — classify and prune the children found by c2t_expand_level(level):
+ *   joint probability P = P_parent * p (Eq. 1), features (P, H of the parent's row, d = level),
+ *   confidence C = F(P, H, d) (Eq. 4), first pruning C >= beta (Alg. 1), second pruning: the F
+ *   survivors with the highest C (ties to the earlier candidate) generate the next layer
+ *   (Sec. 4.2.2); survivors are appended to the tree in candidate order (parent slot, then
+ *   rank) according to cfg.tree_add.  `out` may be NULL.
+ * level == C2T_FINAL — Top-N rerank (Sec. 2.2): keep the root and the N-1 nodes with the
+ *   highest score, the score of a node being the minimum confidence on its root path (ties
+ *   to the lower node id), renumbered in creation order.  `out` is ignored.  Must follow the
+ *   last level pruned (any number of levels <= D).
+ */
+int c2t_prune(c2t_ctx *ctx, int level, const c2t_frontier *out, void *stream);
+
+/* Verification inputs, written by c2t_build_verify.  Caller-owned device arrays, NULL = skip.
+ * Nw = c2t_final_width, W = c2t_mask_words, D = cfg.max_depth. */
+typedef struct {
+  int32_t  *n_nodes;       /* [B]          nodes in the final tree, root included          */
+  int32_t  *tokens;        /* [B, Nw]      token per node; 0 past n_nodes                  */
+  int32_t  *parents;       /* [B, Nw]      parent node id; -1 for the root and past n_nodes */
+  int32_t  *position_ids;  /* [B, Nw]      prefix_len + tree level; 0 past n_nodes         */
+  uint64_t *mask_bits;     /* [B, Nw, W]   bit j of row i set iff j is i or an ancestor of i;
+                                            every node also attends the whole prefix      */
+  int32_t  *retrieve;      /* [B, Nw, D+1] row r: node ids root -> r-th leaf (leaves in
+                                            ascending id order), -1 padded                 */
+  int32_t  *n_leaves;      /* [B]                                                          */
+} c2t_verify;
+
+/* Tree-attention inputs of the final tree (Sec. 2.2).  Must follow c2t_prune(C2T_FINAL). */
+int c2t_build_verify(c2t_ctx *ctx, const c2t_verify *out, void *stream);
+
+typedef struct {
+  int32_t *accept_len;   /* [B]      tau of this step: accepted draft tokens, root excluded */
+  int32_t *path;         /* [B, D+1] accepted node ids, root first, -1 padded               */
+  int32_t *next_token;   /* [B]      the target's greedy token after the last accepted node */
+} c2t_accept_out;
+
+/*
+ * Greedy acceptance over the final tree (Sec. 5 Metrics: the accept length excludes the
+ * target's own token).  target_logits_dev: [B, Nw, V] of cfg.dtype, row (b, i) = target
+ * logits at final node i, element offset b*seq_stride + i*row_stride + v, aligned like the
+ * draft logits; rows i >= n_nodes(b) are never read.  From the root, move to the child
+ * carrying the target's argmax token (ties to the lower id) until none does.
+ * Must follow c2t_prune(C2T_FINAL).
+ */
+int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride,
+               int64_t row_stride, const c2t_accept_out *out, void *stream);
+
+/* Waits for `stream`, then ORs all sequences' status words into *bits_host and, if
+ * per_seq_host is not NULL, copies the B words there.  For tests and debugging. */
+int c2t_status(c2t_ctx *ctx, uint32_t *bits_host, uint32_t *per_seq_host, void *stream);
+
+/*
+ * Read-only device views into the workspace, for inspection and tests.  Tree arrays are
+ * [B, c2t_tree_capacity]; candidate arrays are [B, F*K] and hold the level pruned last
+ * (candidate index = parent slot * K + rank); final arrays are [B, Nw].
+ */
+typedef struct {
+  const int32_t *tree_n;        /* [B]                                                      */
+  const int32_t *tree_token, *tree_parent, *tree_level;
+  const double  *tree_logP;     /* log joint probability                                   */
+  const double  *tree_C;        /* confidence                                              */
+  const double  *tree_Chat;     /* min confidence on the root path (root: +inf)            */
+  const int32_t *cand_n;        /* [B] candidates at the last level                        */
+  const int32_t *cand_token;
+  const double  *cand_lp;       /* log generation probability                              */
+  const double  *cand_logP, *cand_H, *cand_C;
+  const int32_t *cand_flags;    /* bit 0: C >= beta; bit 1: next-layer generator           */
+  const int32_t *frontier_n;    /* [B] generators entering the next expand                 */
+  const int32_t *frontier_node; /* [B, F]                                                  */
+  const int32_t *final_n;       /* [B]                                                     */
+  const int32_t *final_src;     /* [B, Nw] tree id each final node came from               */
+  const int32_t *final_token, *final_parent, *final_level;
+  const int32_t *node_argmax;   /* [B, Nw] target argmax per final node (after c2t_accept) */
+} c2t_view;
+int c2t_get_view(c2t_ctx *ctx, c2t_view *out);
+
+/* Host-side description of a whole decode step fed from host memory. */
+typedef struct {
+  const void *const *draft_logits_host; /* [D] pointers, each [B, F, V] contiguous, pinned  */
+  const void *target_logits_host;       /* [B, Nw, V] contiguous, pinned                    */
+  const int32_t *root_tok_host;         /* [B]                                              */
+  const int32_t *prefix_len_host;       /* [B]                                              */
+  void *draft_stage_dev;                /* device staging, B*F*V elements                   */
+  void *target_stage_dev;               /* device staging, B*Nw*V elements                  */
+  int32_t *int_stage_dev;               /* device staging, c2t_host_step_ints(cfg) int32    */
+  /* results, host */
+  int32_t *n_nodes_host;                /* [B]                                              */
+  int32_t *tokens_host;                 /* [B, Nw]                                          */
+  int32_t *accept_len_host;             /* [B]                                              */
+  int32_t *path_host;                   /* [B, D+1]                                         */
+  int32_t *next_token_host;             /* [B]                                              */
+} c2t_host_step;
+size_t c2t_host_step_ints(const c2t_config *cfg);
+
+/*
+ * One whole decode step (all the calls listed at the top) with inputs and results in HOST
+ * memory: copies each level's draft logits and the target logits to the caller's device
+ * staging buffers on `stream`, runs the step, copies the results back and waits for
+ * `stream`.  Level 0 copies only slot 0 of each sequence (the root's row).  Exists so that
+ * an end-to-end figure including the transfers can be measured through the library.
+ */
+int c2t_decode_step_host(c2t_ctx *ctx, const c2t_host_step *io, void *stream);
+
+/* Number of kernels the context has launched since c2t_init (host-side counter). */
+int64_t c2t_launch_count(const c2t_ctx *ctx);
+
+const char *c2t_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* C2T_H */

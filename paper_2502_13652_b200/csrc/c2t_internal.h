@@ -1,0 +1,105 @@
+// Internal declarations shared by the CUDA translation units of libc2t.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "c2t.h"
+
+namespace c2t {
+
+// ---------------------------------------------------------------- keys ------
+// Total order used everywhere a "largest logit, then lowest token id" decision is taken:
+// key = (orderable(value) << 32) | (0xFFFFFFFF - token).  A larger key wins.  0 = empty.
+
+__host__ __device__ __forceinline__ uint32_t f32_orderable(uint32_t bits) {
+  return bits ^ ((bits & 0x80000000u) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__host__ __device__ __forceinline__ uint32_t f32_from_orderable(uint32_t o) {
+  return o ^ ((o & 0x80000000u) ? 0x80000000u : 0xFFFFFFFFu);
+}
+__device__ __forceinline__ unsigned long long make_key(float x, uint32_t tok) {
+  return ((unsigned long long)f32_orderable(__float_as_uint(x)) << 32) | (0xFFFFFFFFu - tok);
+}
+__device__ __forceinline__ float key_value(unsigned long long k) {
+  return __uint_as_float(f32_from_orderable((uint32_t)(k >> 32)));
+}
+__device__ __forceinline__ int32_t key_token(unsigned long long k) {
+  return (int32_t)(0xFFFFFFFFu - (uint32_t)k);
+}
+
+// Logits of -inf are read as the lowest finite value of the storage type, so that
+// "probability zero" never produces inf - inf or 0 * inf in the running sums.
+constexpr float kNegInfAsFinite = -3.38e38f;   // anything at or below this was -inf (or as good as)
+
+// ---------------------------------------------------------------- vocab pass -
+
+constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass
+constexpr int kPassCtasPerSm = 2;
+constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors than this
+
+// What one launch of the vocabulary pass derived from the device-side row counts.
+struct PassInfo {
+  int32_t n_rows;       // active rows
+  int32_t vec_per_row;  // 16-byte vectors per row (last one may be ragged)
+  int64_t span;         // vectors per CTA
+};
+
+struct PassParams {
+  const void *logits;
+  int64_t seq_stride, row_stride;   // elements
+  int32_t V, K, B;
+  int32_t rows_per_seq_max;         // F (draft) or Nw (target)
+  const int32_t *counts;            // [B] active rows per sequence, device
+  int32_t max_splits;               // partial slots per row
+  PassInfo *info;                   // written by CTA 0
+  // expand: per (row, split) partial
+  float4 *part_stats;               // {m_ref, S, T, n_keys as int bits}
+  unsigned long long *part_keys;    // [.. * K] sorted descending, 0-padded
+  // argmax: per (row, split) best key
+  unsigned long long *part_best;
+};
+
+int max_splits_for(int vocab, int elem_bytes, int grid);
+
+cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
+cudaError_t launch_argmax_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
+
+// ---------------------------------------------------------------- tree state -
+
+struct TreeState {
+  int32_t B, V, K, F, D, N, Nw, W, cap, hidden, classifier, tree_add, max_splits, max_splits_tgt;
+  float beta;
+  // frontier, double buffered by level parity
+  int32_t *frontier_n[2];      // [B]
+  int32_t *frontier_node[2];   // [B, F]
+  // tree
+  int32_t *tree_n;             // [B]
+  int32_t *tree_token, *tree_parent, *tree_level;   // [B, cap]
+  double *tree_logP, *tree_C, *tree_Chat;           // [B, cap]
+  int32_t *remap;              // [B, cap] scratch of the rerank
+  // candidates of the last level
+  int32_t *cand_n;             // [B]
+  int32_t *cand_token, *cand_flags;                 // [B, F*K]
+  double *cand_lp, *cand_logP, *cand_H, *cand_C;    // [B, F*K]
+  // final tree
+  int32_t *final_n;            // [B]
+  int32_t *final_src, *final_token, *final_parent, *final_level;   // [B, Nw]
+  int32_t *node_argmax;        // [B, Nw]
+  int32_t *root_tok, *prefix_len;                   // [B]
+  uint32_t *status;            // [B]
+  PassInfo *info_draft, *info_target;
+  float4 *part_stats;
+  unsigned long long *part_keys;
+  unsigned long long *part_best;
+  float *w1, *b1, *w2, *b2;
+};
+
+cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
+                              cudaStream_t s);
+cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s);
+cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s);
+cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s);
+cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s);
+
+}  // namespace c2t

@@ -1,0 +1,519 @@
+// Per-sequence kernels: classification and pruning of a level, the Top-N rerank, the
+// verification inputs and the acceptance walk.  One CTA per sequence; all of this is
+// O(F*K) or O(tree) work per sequence, done in double precision where it is floating point.
+#include "c2t_internal.h"
+
+namespace c2t {
+namespace {
+
+constexpr int kTreeThreads = 256;
+constexpr int kTreeWarps = kTreeThreads / 32;
+constexpr int kMaxCand = C2T_MAX_TOPK * C2T_MAX_FRONTIER;   // 1024
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(kFull, v, o);
+  return __shfl_sync(kFull, v, 0);
+}
+
+// Exclusive scan of one int per thread over the CTA; returns the exclusive prefix, *total = sum.
+__device__ int block_exclusive_scan(int v, int *s_warp /*[kTreeWarps+1]*/, int *total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(kFull, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    for (int w = 0; w < kTreeWarps; ++w) { int t = s_warp[w]; s_warp[w] = run; run += t; }
+    s_warp[kTreeWarps] = run;
+  }
+  __syncthreads();
+  *total = s_warp[kTreeWarps];
+  return s_warp[warp] + inc - v;
+}
+
+__global__ void begin_step_kernel(TreeState t, const int32_t *root_tok, const int32_t *prefix_len) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= t.B) return;
+  const size_t o = (size_t)b * t.cap;
+  t.tree_n[b] = 1;
+  t.tree_token[o] = root_tok[b];
+  t.tree_parent[o] = -1;
+  t.tree_level[o] = 0;
+  t.tree_logP[o] = 0.0;
+  t.tree_C[o] = 1.0;
+  t.tree_Chat[o] = INFINITY;
+  t.frontier_n[0][b] = 1;
+  t.frontier_n[1][b] = 0;
+  t.frontier_node[0][(size_t)b * t.F] = 0;
+  t.cand_n[b] = 0;
+  t.final_n[b] = 0;
+  t.root_tok[b] = root_tok[b];
+  t.prefix_len[b] = prefix_len[b];
+  t.status[b] = 0u;
+}
+
+// ---------------------------------------------------------------- a level ---
+
+// Confidence of one child (Eq. 4): two-layer FFN on (P, H, d), ReLU, sigmoid.
+__device__ double classify(const TreeState &t, const float *s_w, double P, double H, double d) {
+  const float *w1 = s_w, *b1 = s_w + 3 * C2T_MAX_HIDDEN, *w2 = b1 + C2T_MAX_HIDDEN, *b2 = w2 + C2T_MAX_HIDDEN;
+  double z = (double)b2[0];
+  for (int k = 0; k < t.hidden; ++k) {
+    double a = (double)b1[k] + (double)w1[3 * k] * P + (double)w1[3 * k + 1] * H + (double)w1[3 * k + 2] * d;
+    if (a < 0.0) a = 0.0;
+    z += (double)w2[k] * a;
+  }
+  return 1.0 / (1.0 + exp(-z));
+}
+
+__global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, int level, c2t_frontier out) {
+  __shared__ float s_w[5 * C2T_MAX_HIDDEN + 4];
+  __shared__ double s_rowM[C2T_MAX_FRONTIER], s_rowL[C2T_MAX_FRONTIER], s_rowH[C2T_MAX_FRONTIER];
+  __shared__ int s_rowfault[C2T_MAX_FRONTIER];
+  __shared__ float s_x[kMaxCand];
+  __shared__ int s_tok[kMaxCand];
+  __shared__ double s_C[kMaxCand];
+  __shared__ unsigned char s_keep[kMaxCand], s_sel[kMaxCand];
+  __shared__ int s_scan[kTreeWarps + 1];
+  __shared__ int s_misc[2];
+
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = t.K, F = t.F;
+  const int cur = level & 1, nxt = cur ^ 1;
+  int n = t.frontier_n[cur][b];
+  n = n < 0 ? 0 : (n > F ? F : n);
+  const size_t cbase = (size_t)b * F * K;
+
+  if (n == 0) {                                   // the loop of Alg. 1 has ended for this sequence
+    if (tid == 0) {
+      t.frontier_n[nxt][b] = 0;
+      t.cand_n[b] = 0;
+      if (out.count) out.count[b] = 0;
+    }
+    return;
+  }
+  // rows of earlier sequences
+  {
+    int part = 0;
+    for (int i = tid; i < b; i += kTreeThreads) {
+      int c = t.frontier_n[cur][i];
+      part += c < 0 ? 0 : (c > F ? F : c);
+    }
+    int total;
+    block_exclusive_scan(part, s_scan, &total);
+    if (tid == 0) s_misc[0] = total;
+  }
+  if (t.classifier == C2T_CLS_MLP) {
+    for (int i = tid; i < 3 * t.hidden; i += kTreeThreads) s_w[i] = t.w1[i];
+    for (int i = tid; i < t.hidden; i += kTreeThreads) {
+      s_w[3 * C2T_MAX_HIDDEN + i] = t.b1[i];
+      s_w[4 * C2T_MAX_HIDDEN + i] = t.w2[i];
+    }
+    if (tid == 0) s_w[5 * C2T_MAX_HIDDEN] = t.b2[0];
+  }
+  __syncthreads();
+  const int row_off = s_misc[0];
+  const PassInfo info = *t.info_draft;
+
+  // ---- phase 1: one warp per row merges that row's partial records
+  for (int j = warp; j < n; j += kTreeWarps) {
+    const int a = row_off + j;
+    const long long first_vec = (long long)a * info.vec_per_row;
+    const int c_first = (int)(first_vec / info.span);
+    const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
+    int n_splits = c_last - c_first + 1;
+    if (n_splits > t.max_splits) n_splits = t.max_splits;
+    const size_t slot0 = (size_t)a * t.max_splits;
+    const int n_keys = n_splits * K;
+
+    // the row maximum is the largest key of any partial
+    unsigned long long top = 0ull;
+    for (int i = lane; i < n_splits; i += 32) {
+      unsigned long long k0 = t.part_keys[(slot0 + i) * K];
+      top = k0 > top ? k0 : top;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      unsigned long long other = __shfl_xor_sync(kFull, top, o);
+      top = other > top ? other : top;
+    }
+    const double M = (double)key_value(top);
+
+    // fp32 tails of every split, rescaled to M
+    double S = 0.0, T = 0.0;
+    for (int i = lane; i < n_splits; i += 32) {
+      float4 st = t.part_stats[slot0 + i];
+      double Ss = (double)st.y, Ts = (double)st.z;
+      if (Ss != 0.0 || Ts != 0.0) {               // (NaN passes this test and poisons the sums)
+        double d = (double)st.x - M;
+        double f = exp(d);
+        S += Ss * f;
+        T += f * (Ts + d * Ss);
+      }
+    }
+    // exact keys: rank them; all but the row maximum join the sums; the K best become candidates
+    for (int i = lane; i < n_keys; i += 32) {
+      const unsigned long long key = t.part_keys[slot0 * K + i];
+      if (key == 0ull) continue;
+      const int tok = key_token(key);
+      if (tok >= t.V) continue;                   // padding of a ragged last vector
+      int rank = 0;
+      for (int r = 0; r < n_keys; ++r) {
+        unsigned long long other = t.part_keys[slot0 * K + r];
+        rank += (other > key) && (key_token(other) < t.V);
+      }
+      const float x = key_value(key);
+      if (key != top && x > kNegInfAsFinite) {
+        double d = (double)x - M;
+        double e = exp(d);
+        S += e;
+        T += e * d;
+      }
+      if (rank < K) { s_x[j * K + rank] = x; s_tok[j * K + rank] = tok; }
+    }
+    S = warp_sum(S);
+    T = warp_sum(T);
+    // candidates that do not exist (fewer than K tokens in the vocabulary)
+    int n_valid = 0;
+    for (int i = lane; i < n_keys; i += 32) {
+      unsigned long long key = t.part_keys[slot0 * K + i];
+      n_valid += (key != 0ull && key_token(key) < t.V);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n_valid += __shfl_xor_sync(kFull, n_valid, o);
+    for (int r = (n_valid < K ? n_valid : K) + lane; r < K; r += 32) { s_x[j * K + r] = -INFINITY; s_tok[j * K + r] = -1; }
+
+    if (lane == 0) {
+      uint32_t fault = 0;
+      const float top_x = key_value(top);
+      if (top == 0ull || top_x <= kNegInfAsFinite) fault |= C2T_ST_ALL_NEGINF;
+      else if (top_x == INFINITY) fault |= C2T_ST_POSINF_LOGIT;
+      else if (S != S || T != T || isinf(S)) fault |= C2T_ST_NAN_LOGIT;
+      const double L = log1p(S);                  // ln sum_v e^(x_v - M); the maximum contributes the 1
+      s_rowM[j] = M;
+      s_rowL[j] = L;
+      s_rowH[j] = L - T / (1.0 + S);              // Eq. 2 with natural log
+      s_rowfault[j] = (int)fault;
+      if (fault) atomicOr(&t.status[b], fault);
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 2: features and confidence, one thread per candidate child
+  const int nc = n * K;
+  for (int c = tid; c < nc; c += kTreeThreads) {
+    const int j = c / K;
+    const int f = t.frontier_node[cur][(size_t)b * F + j];
+    const int tok = s_tok[c];
+    const float x = s_x[c];
+    const bool ok = tok >= 0 && !s_rowfault[j];
+    const double lp = (x > kNegInfAsFinite) ? ((double)x - s_rowM[j]) - s_rowL[j] : -INFINITY;
+    const double logP = t.tree_logP[(size_t)b * t.cap + f] + lp;           // Eq. 1 in log space
+    const double P = exp(logP);
+    const double H = s_rowH[j];
+    double C;
+    if (!ok) C = NAN;
+    else if (t.classifier == C2T_CLS_IDENTITY_JOINT) C = P;
+    else C = classify(t, s_w, P, H, (double)level);
+    const bool keep = ok && C >= (double)t.beta;                            // first pruning
+    s_C[c] = C;
+    s_keep[c] = keep;
+    s_sel[c] = keep;
+    t.cand_token[cbase + c] = tok;
+    t.cand_lp[cbase + c] = ok ? lp : NAN;
+    t.cand_logP[cbase + c] = ok ? logP : NAN;
+    t.cand_H[cbase + c] = ok ? H : NAN;
+    t.cand_C[cbase + c] = C;
+  }
+  __syncthreads();
+
+  // ---- phase 3: second pruning, the F survivors that come first under (C desc, index asc)
+  int my_keep = 0;
+  for (int c = tid; c < nc; c += kTreeThreads) my_keep += s_keep[c];
+  int n_keep;
+  block_exclusive_scan(my_keep, s_scan, &n_keep);
+  if (n_keep > F) {
+    for (int c = tid; c < nc; c += kTreeThreads) {
+      if (!s_keep[c]) continue;
+      const double Cc = s_C[c];
+      int rank = 0;
+      for (int o = 0; o < nc; ++o)
+        if (s_keep[o]) rank += (s_C[o] > Cc) || (s_C[o] == Cc && o < c);
+      s_sel[c] = rank < F;
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 4: stable compaction in candidate order; append to the tree, emit the frontier
+  const int per = (nc + kTreeThreads - 1) / kTreeThreads;      // consecutive candidates per thread
+  const int c0 = tid * per, c1 = (c0 + per < nc) ? c0 + per : nc;
+  const bool add_all = t.tree_add == C2T_ADD_ALL_SURVIVORS;
+  int n_add = 0, n_sel = 0;
+  for (int c = c0; c < c1; ++c) { n_add += add_all ? s_keep[c] : s_sel[c]; n_sel += s_sel[c]; }
+  int tot_add, tot_sel;
+  int off_add = block_exclusive_scan(n_add, s_scan, &tot_add);
+  int off_sel = block_exclusive_scan(n_sel, s_scan, &tot_sel);
+  const int base = t.tree_n[b];
+  const bool overflow = base + tot_add > t.cap;
+  const size_t tb = (size_t)b * t.cap;
+  for (int c = c0; c < c1; ++c) {
+    const bool add = add_all ? s_keep[c] : s_sel[c];
+    int flags = (s_keep[c] ? 1 : 0) | (s_sel[c] ? 2 : 0);
+    t.cand_flags[cbase + c] = flags;
+    if (!add) continue;
+    const int id = base + off_add++;
+    if (id < t.cap) {
+      const int j = c / K;
+      const int f = t.frontier_node[cur][(size_t)b * F + j];
+      t.tree_token[tb + id] = s_tok[c];
+      t.tree_parent[tb + id] = f;
+      t.tree_level[tb + id] = level + 1;
+      t.tree_logP[tb + id] = t.cand_logP[cbase + c];
+      t.tree_C[tb + id] = s_C[c];
+      const double ch = t.tree_Chat[tb + f];
+      t.tree_Chat[tb + id] = s_C[c] < ch ? s_C[c] : ch;
+    }
+    if (s_sel[c] && !overflow) {
+      const int slot = off_sel++;
+      t.frontier_node[nxt][(size_t)b * F + slot] = id;
+      if (out.token) out.token[(size_t)b * F + slot] = s_tok[c];
+      if (out.node_id) out.node_id[(size_t)b * F + slot] = id;
+      if (out.parent_slot) out.parent_slot[(size_t)b * F + slot] = c / K;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const int next_n = overflow ? 0 : tot_sel;
+    t.tree_n[b] = overflow ? t.cap : base + tot_add;
+    t.frontier_n[nxt][b] = next_n;
+    t.cand_n[b] = nc;
+    if (out.count) out.count[b] = next_n;
+    if (overflow) atomicOr(&t.status[b], C2T_ST_TREE_OVERFLOW);
+  }
+}
+
+// ---------------------------------------------------------------- rerank ----
+
+// Top-N rerank (Sec. 2.2): root + the N-1 nodes first under (Chat desc, id asc), renumbered
+// in id order.  Chat never exceeds the parent's and parents have lower ids, so the kept set
+// is closed under "parent of".
+__global__ void __launch_bounds__(kTreeThreads) final_prune_kernel(TreeState t) {
+  __shared__ int s_scan[kTreeWarps + 1];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  int n = t.tree_n[b];
+  n = n > t.cap ? t.cap : n;
+  const size_t tb = (size_t)b * t.cap, fb = (size_t)b * t.Nw;
+  const double *chat = t.tree_Chat + tb;
+  int32_t *remap = t.remap + tb;
+  const bool all = (t.N <= 0 || n <= t.N);
+
+  int run = 0;     // nodes kept so far (ids below the chunk)
+  for (int base = 0; base < n; base += kTreeThreads) {
+    const int i = base + tid;
+    int keep = 0;
+    if (i < n) {
+      if (all || i == 0) keep = 1;
+      else {
+        const double ci = chat[i];
+        int rank = 0;
+        for (int o = 1; o < n; ++o) {
+          const double co = __ldg(&chat[o]);
+          rank += (co > ci) || (co == ci && o < i);
+        }
+        keep = rank < t.N - 1;
+      }
+    }
+    int total;
+    const int off = block_exclusive_scan(keep, s_scan, &total);
+    if (i < n) remap[i] = keep ? run + off : -1;
+    run += total;
+  }
+  __syncthreads();
+  const int n_final = run > t.Nw ? t.Nw : run;
+  for (int i = tid; i < n; i += kTreeThreads) {
+    const int m = remap[i];
+    if (m < 0 || m >= t.Nw) continue;
+    const int par = t.tree_parent[tb + i];
+    t.final_src[fb + m] = i;
+    t.final_token[fb + m] = t.tree_token[tb + i];
+    t.final_parent[fb + m] = par < 0 ? -1 : remap[par];
+    t.final_level[fb + m] = t.tree_level[tb + i];
+  }
+  for (int m = n_final + tid; m < t.Nw; m += kTreeThreads) {
+    t.final_src[fb + m] = -1;
+    t.final_token[fb + m] = 0;
+    t.final_parent[fb + m] = -1;
+    t.final_level[fb + m] = 0;
+  }
+  if (tid == 0) t.final_n[b] = n_final;
+}
+
+// ---------------------------------------------------------------- verify ----
+
+__global__ void __launch_bounds__(kTreeThreads) build_verify_kernel(TreeState t, c2t_verify out) {
+  __shared__ int s_has_child[C2T_MAX_BUDGET > C2T_MAX_TREE ? C2T_MAX_BUDGET : C2T_MAX_TREE];
+  __shared__ int s_scan[kTreeWarps + 1];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int n = t.final_n[b], Nw = t.Nw, W = t.W, width = t.D + 1;
+  const size_t fb = (size_t)b * Nw;
+  const int32_t *parent = t.final_parent + fb, *level = t.final_level + fb;
+  const int prefix = t.prefix_len[b];
+
+  for (int i = tid; i < Nw; i += kTreeThreads) s_has_child[i] = 0;
+  __syncthreads();
+  for (int i = tid; i < n; i += kTreeThreads)
+    if (parent[i] >= 0) s_has_child[parent[i]] = 1;
+  __syncthreads();
+
+  for (int i = tid; i < Nw; i += kTreeThreads) {
+    if (out.tokens) out.tokens[fb + i] = i < n ? t.final_token[fb + i] : 0;
+    if (out.parents) out.parents[fb + i] = i < n ? parent[i] : -1;
+    if (out.position_ids) out.position_ids[fb + i] = i < n ? prefix + level[i] : 0;
+    if (out.mask_bits) {
+      uint64_t *row = out.mask_bits + (fb + i) * W;
+      for (int w = 0; w < W; ++w) row[w] = 0ull;
+      if (i < n)
+        for (int a = i, g = 0; a >= 0 && g <= t.D + 1; a = parent[a], ++g) row[a >> 6] |= 1ull << (a & 63);
+    }
+    if (out.retrieve) {
+      int32_t *row = out.retrieve + (fb + i) * width;
+      for (int k = 0; k < width; ++k) row[k] = -1;
+    }
+  }
+  __syncthreads();
+  // leaves in ascending id order
+  int run = 0;
+  for (int base = 0; base < n; base += kTreeThreads) {
+    const int i = base + tid;
+    const int leaf = (i < n && !s_has_child[i]) ? 1 : 0;
+    int total;
+    const int off = block_exclusive_scan(leaf, s_scan, &total);
+    if (leaf && out.retrieve) {
+      int32_t *row = out.retrieve + (fb + run + off) * width;
+      for (int a = i, g = 0; a >= 0 && g <= t.D + 1; a = parent[a], ++g) {
+        const int l = level[a];
+        if (l >= 0 && l < width) row[l] = a;
+      }
+    }
+    run += total;
+  }
+  if (tid == 0) {
+    if (out.n_nodes) out.n_nodes[b] = n;
+    if (out.n_leaves) out.n_leaves[b] = run;
+  }
+}
+
+// ---------------------------------------------------------------- accept ----
+
+__global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, c2t_accept_out out) {
+  __shared__ int s_misc[1];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = t.final_n[b], Nw = t.Nw, width = t.D + 1;
+  const size_t fb = (size_t)b * Nw;
+  const PassInfo info = *t.info_target;
+
+  // rows of earlier sequences in the argmax pass
+  {
+    __shared__ int s_scan[kTreeWarps + 1];
+    int part = 0;
+    for (int i = tid; i < b; i += kTreeThreads) {
+      int c = t.final_n[i];
+      part += c < 0 ? 0 : (c > Nw ? Nw : c);
+    }
+    int total;
+    block_exclusive_scan(part, s_scan, &total);
+    if (tid == 0) s_misc[0] = total;
+    __syncthreads();
+  }
+  const int row_off = s_misc[0];
+  // target argmax per node: best key over the row's partials
+  for (int i = tid; i < Nw; i += kTreeThreads) {
+    int tok = -1;
+    if (i < n) {
+      const int a = row_off + i;
+      const long long first_vec = (long long)a * info.vec_per_row;
+      const int c_first = (int)(first_vec / info.span);
+      const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
+      int n_splits = c_last - c_first + 1;
+      if (n_splits > t.max_splits_tgt) n_splits = t.max_splits_tgt;
+      unsigned long long best = 0ull;
+      for (int s = 0; s < n_splits; ++s) {
+        unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + s];
+        best = k > best ? k : best;
+      }
+      tok = best ? key_token(best) : -1;
+    }
+    t.node_argmax[fb + i] = tok;
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  // greedy walk by one warp
+  const int32_t *parent = t.final_parent + fb, *token = t.final_token + fb;
+  int cur = 0, len = 0;
+  if (out.path && lane < width) out.path[(size_t)b * width + lane] = lane == 0 ? 0 : -1;
+  for (int w = 32 + lane; out.path && w < width; w += 32) out.path[(size_t)b * width + w] = -1;
+  __syncwarp();
+  while (n > 0 && len + 1 < width) {
+    const int want = t.node_argmax[fb + cur];
+    int found = 0x7FFFFFFF;
+    for (int c = cur + 1 + lane; c < n; c += 32)
+      if (parent[c] == cur && token[c] == want) { found = c; break; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      int other = __shfl_xor_sync(kFull, found, o);
+      found = other < found ? other : found;
+    }
+    if (found == 0x7FFFFFFF) break;
+    cur = found;
+    ++len;
+    if (lane == 0 && out.path) out.path[(size_t)b * width + len] = cur;
+  }
+  if (lane == 0) {
+    if (out.accept_len) out.accept_len[b] = len;
+    if (out.next_token) out.next_token[b] = n > 0 ? t.node_argmax[fb + cur] : -1;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
+                              cudaStream_t s) {
+  begin_step_kernel<<<(t.B + 127) / 128, 128, 0, s>>>(t, root_tok, prefix_len);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s) {
+  c2t_frontier o = {nullptr, nullptr, nullptr, nullptr};
+  if (out) o = *out;
+  prune_level_kernel<<<t.B, kTreeThreads, 0, s>>>(t, level, o);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s) {
+  final_prune_kernel<<<t.B, kTreeThreads, 0, s>>>(t);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s) {
+  c2t_verify o = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (out) o = *out;
+  build_verify_kernel<<<t.B, kTreeThreads, 0, s>>>(t, o);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s) {
+  c2t_accept_out o = {nullptr, nullptr, nullptr};
+  if (out) o = *out;
+  accept_walk_kernel<<<t.B, kTreeThreads, 0, s>>>(t, o);
+  return cudaGetLastError();
+}
+
+}  // namespace c2t

@@ -1,0 +1,243 @@
+"""Helpers shared by the GPU parity tests: run the library and the oracle on the same bytes
+and compare them element by element.
+
+Tolerances (relative, on probabilities, entropies and confidences): 1e-5 for fp32 logits,
+2e-3 for bf16 logits.  Everything integer (tokens, kept sets, parents, masks, positions,
+retrieve rows, accept lengths) must be identical.  A sequence in which the oracle itself sits
+within 1e-6 of a decision boundary (confidence vs. threshold, F-th vs. (F+1)-th survivor,
+budget cut) is a "near tie": it is counted and, from that level on, excluded from the exact
+comparison if and only if the two sides actually disagree.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+import c2t_inputs
+import oracle
+import paper_2502_13652_b200 as c2t
+
+RTOL = {torch.float32: 1e-5, torch.bfloat16: 2e-3}
+NEAR = 1e-6
+
+
+def make_configs(B, V, D, K, F, N, beta, dtype, classifier="mlp", hidden=16, tree_add="frontier",
+                 wseed=0, wstd=0.1, weights=None):
+    w1, b1, w2, b2 = weights if weights is not None else c2t_inputs.classifier_weights(hidden, seed=wseed, std=wstd)
+    ocfg = oracle.OracleConfig(
+        vocab=V, dtype=oracle.BF16 if dtype == torch.bfloat16 else oracle.F32, max_depth=D, topk=K,
+        frontier_cap=F, budget=N, threshold=beta,
+        classifier=oracle.CLS_MLP if classifier == "mlp" else oracle.CLS_IDENTITY_JOINT,
+        hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
+        tree_add=oracle.ADD_FRONTIER if tree_add == "frontier" else oracle.ADD_ALL_SURVIVORS)
+    gcfg = c2t.Config(
+        batch=B, vocab=V, dtype=c2t.BF16 if dtype == torch.bfloat16 else c2t.F32, max_depth=D, topk=K,
+        frontier_cap=F, budget=N, threshold=beta,
+        classifier=c2t.CLS_MLP if classifier == "mlp" else c2t.CLS_IDENTITY_JOINT,
+        hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
+        tree_add=c2t.ADD_FRONTIER if tree_add == "frontier" else c2t.ADD_ALL_SURVIVORS)
+    return ocfg, gcfg
+
+
+def gen_inputs(B, V, D, F, Nw, dtype, step=0, scale=4.0, device="cpu", seq_base=0):
+    draft = [c2t_inputs.draft_logits(B, F, V, step, l, dtype, scale, device=device, seq_base=seq_base)
+             for l in range(D)]
+    target = c2t_inputs.target_logits(B, Nw, V, step, dtype, scale, device=device, seq_base=seq_base)
+    root = c2t_inputs.root_tokens(B, V, step, seq_base)
+    prefix = c2t_inputs.prefix_lengths(B, seq_base=seq_base)
+    return draft, target, root, prefix
+
+
+@dataclass
+class Report:
+    sequences: int = 0
+    near_tie_sequences: int = 0
+    diverged_sequences: int = 0
+    max_rel_p: float = 0.0
+    max_rel_H: float = 0.0
+    max_rel_C: float = 0.0
+    kept_nodes: list = field(default_factory=list)
+    accept_len: list = field(default_factory=list)
+
+    def line(self) -> str:
+        return (f"seq={self.sequences} near_tie={self.near_tie_sequences} diverged={self.diverged_sequences} "
+                f"max_rel p={self.max_rel_p:.2e} H={self.max_rel_H:.2e} C={self.max_rel_C:.2e} "
+                f"mean_nodes={np.mean(self.kept_nodes) if self.kept_nodes else 0:.1f} "
+                f"mean_tau={np.mean(self.accept_len) if self.accept_len else 0:.2f}")
+
+
+def _rel(a: np.ndarray, b: np.ndarray) -> float:
+    """max |a-b| / |b| over finite entries (0 where both are 0)."""
+    a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
+    if a.size == 0:
+        return 0.0
+    den = np.maximum(np.abs(b), 1e-300)
+    r = np.abs(a - b) / den
+    r[(a == b)] = 0.0
+    return float(np.nanmax(r)) if np.isfinite(r).any() else 0.0
+
+
+def _near_tie_at_level(L, l, F, beta) -> bool:
+    n = int(L.n_cand[l])
+    Cv = L.C[l, :n]
+    if n == 0:
+        return False
+    if np.any(np.abs(Cv - beta) <= NEAR):
+        return True
+    surv = np.sort(Cv[L.keep[l, :n] == 1])[::-1]
+    if len(surv) > F and abs(surv[F - 1] - surv[F]) <= NEAR * max(abs(surv[F - 1]), 1e-300):
+        # an exact tie is decided by candidate order on both sides; only a near-but-unequal pair is fragile
+        return surv[F - 1] != surv[F]
+    return False
+
+
+def _near_tie_budget(tree, N) -> bool:
+    if N <= 0 or tree.n <= N:
+        return False
+    ch = np.sort(tree.Chat[1:tree.n])[::-1]
+    a, b = ch[N - 2], ch[N - 1]
+    return a != b and abs(a - b) <= NEAR * max(abs(a), 1e-300)
+
+
+def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, ctx=None,
+                    draft_dev=None, target_dev=None, check_levels=True) -> Report:
+    """Runs one decode step on the GPU (level by level) and on the oracle; asserts parity.
+
+    draft_cpu: list of D tensors [B,F,V] on CPU (or None when `seqs` rows are pulled from
+    draft_dev); seqs: sequences the oracle checks (default all)."""
+    dtype = gcfg.torch_dtype
+    rtol = RTOL[dtype]
+    B, D, F, K = gcfg.batch, gcfg.max_depth, gcfg.frontier_cap, gcfg.topk
+    own = ctx is None
+    if own:
+        ctx = c2t.Context(gcfg)
+    dev = ctx.device
+    if draft_dev is None:
+        draft_dev = [t.to(dev) for t in draft_cpu]
+        target_dev = target_cpu.to(dev)
+    seqs = list(range(B)) if seqs is None else list(seqs)
+    beta = float(np.float32(gcfg.threshold))
+
+    # oracle, one sequence at a time
+    orc = {}
+    for b in seqs:
+        if draft_cpu is not None:
+            lg = torch.stack([draft_cpu[l][b] for l in range(D)])
+            tg = target_cpu[b]
+        else:
+            lg = torch.stack([draft_dev[l][b].cpu() for l in range(D)])
+            tg = target_dev[b].cpu()
+        tree, L = oracle.build_tree(ocfg, lg, int(root[b]))
+        ft = oracle.final_prune(tree, ocfg.budget)
+        ver = oracle.build_verify(ft, int(prefix[b]), ctx.Nw, D + 1)
+        acc = oracle.accept(ft, tg[:max(ft.n, 1)], D + 1)
+        orc[b] = (tree, L, ft, ver, acc)
+
+    rep = Report(sequences=len(seqs))
+    near = {b: False for b in seqs}
+    diverged = {b: False for b in seqs}
+
+    root_d = root.to(dev); prefix_d = prefix.to(dev)
+    ctx.c2t_begin_step(root_d, prefix_d)
+    for l in range(D):
+        ctx.c2t_expand_level(l, draft_dev[l])
+        ctx.c2t_prune(l)
+        if not check_levels:
+            continue
+        view = ctx.c2t_get_view()
+        torch.cuda.synchronize()
+        g_n = view["cand_n"].cpu().numpy()
+        g_tok = view["cand_token"].cpu().numpy(); g_flags = view["cand_flags"].cpu().numpy()
+        g_lp = view["cand_lp"].cpu().numpy(); g_logP = view["cand_logP"].cpu().numpy()
+        g_H = view["cand_H"].cpu().numpy(); g_C = view["cand_C"].cpu().numpy()
+        g_fn = view["frontier_n"].cpu().numpy(); g_fnode = view["frontier_node"].cpu().numpy()
+        e_cnt = ctx.frontier["count"].cpu().numpy(); e_tok = ctx.frontier["token"].cpu().numpy()
+        e_node = ctx.frontier["node_id"].cpu().numpy(); e_ps = ctx.frontier["parent_slot"].cpu().numpy()
+        for b in seqs:
+            if diverged[b]:
+                continue
+            tree, L, *_ = orc[b]
+            n = int(L.n_cand[l])
+            near[b] = near[b] or _near_tie_at_level(L, l, F, beta)
+            assert g_n[b] == n, f"level {l} seq {b}: candidate count {g_n[b]} != {n}"
+            if n == 0:
+                assert g_fn[b] == 0
+                continue
+            assert np.array_equal(g_tok[b, :n], L.tok[l, :n]), f"level {l} seq {b}: top-K tokens differ"
+            rp = _rel(np.exp(g_lp[b, :n]), np.exp(L.lp[l, :n]))
+            rP = _rel(np.exp(g_logP[b, :n]), np.exp(L.logP[l, :n]))
+            rH = _rel(g_H[b, :n], L.H[l, :n]); rC = _rel(g_C[b, :n], L.C[l, :n])
+            rep.max_rel_p = max(rep.max_rel_p, rp, rP); rep.max_rel_H = max(rep.max_rel_H, rH)
+            rep.max_rel_C = max(rep.max_rel_C, rC)
+            assert rp <= rtol and rP <= rtol, f"level {l} seq {b}: probability error {rp:.2e}/{rP:.2e}"
+            assert rH <= rtol, f"level {l} seq {b}: entropy error {rH:.2e}"
+            assert rC <= rtol, f"level {l} seq {b}: confidence error {rC:.2e}"
+            o_flags = L.keep[l, :n] | (L.next[l, :n] << 1)
+            same = np.array_equal(g_flags[b, :n], o_flags)
+            if not same and near[b]:
+                diverged[b] = True
+                continue
+            assert same, f"level {l} seq {b}: keep/next flags differ"
+            nn = int(L.n_frontier[l + 1])
+            assert g_fn[b] == nn and e_cnt[b] == nn
+            assert np.array_equal(g_fnode[b, :nn], L.frontier_node[l + 1, :nn])
+            assert np.array_equal(e_node[b, :nn], L.frontier_node[l + 1, :nn])
+            sel = np.nonzero(L.next[l, :n])[0]
+            assert np.array_equal(e_tok[b, :nn], L.tok[l, sel])
+            assert np.array_equal(e_ps[b, :nn], sel // K)
+
+    ctx.c2t_prune(c2t.FINAL)
+    ctx.c2t_build_verify()
+    ctx.c2t_accept(target_dev)
+    bits, per = ctx.c2t_status()
+    view = {k: v.cpu().numpy() for k, v in ctx.c2t_get_view().items()}
+    ver_g = {k: v.cpu().numpy() for k, v in ctx.verify.items()}
+    acc_g = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+    for b in seqs:
+        tree, L, ft, ver, acc = orc[b]
+        near[b] = near[b] or _near_tie_budget(tree, ocfg.budget)
+        if not check_levels and not diverged[b]:
+            for l in range(D):
+                near[b] = near[b] or _near_tie_at_level(L, l, F, beta)
+        rep.kept_nodes.append(ft.n); rep.accept_len.append(acc.accept_len)
+        if diverged[b]:
+            continue
+        ok = True
+        n = tree.n
+        ok &= view["tree_n"][b] == n
+        if ok:
+            ok &= np.array_equal(view["tree_token"][b, :n], tree.tok[:n])
+            ok &= np.array_equal(view["tree_parent"][b, :n], tree.parent[:n])
+            ok &= np.array_equal(view["tree_level"][b, :n], tree.level[:n])
+        m = ft.n
+        ok &= view["final_n"][b] == m and ver_g["n_nodes"][b] == m
+        if ok:
+            ok &= np.array_equal(view["final_src"][b, :m], ft.src[:m])
+            ok &= np.array_equal(ver_g["tokens"][b], np.where(np.arange(ctx.Nw) < m, ft.tok[:ctx.Nw], 0))
+            ok &= np.array_equal(ver_g["parents"][b], np.where(np.arange(ctx.Nw) < m, ft.parent[:ctx.Nw], -1))
+            ok &= np.array_equal(ver_g["position_ids"][b], ver.position_ids)
+            ok &= np.array_equal(ver_g["mask_bits"][b].view(np.uint64), ver.mask)
+            ok &= np.array_equal(ver_g["retrieve"][b], ver.retrieve)
+            ok &= ver_g["n_leaves"][b] == ver.n_leaves
+            ok &= np.array_equal(view["node_argmax"][b, :m], acc.node_argmax[:m])
+            ok &= acc_g["accept_len"][b] == acc.accept_len
+            ok &= np.array_equal(acc_g["path"][b], acc.path)
+            ok &= acc_g["next_token"][b] == acc.next_token
+        if not ok and near[b]:
+            diverged[b] = True
+            continue
+        assert ok, f"seq {b}: final tree / verify inputs / accept result differ from the oracle"
+        if n > 1:
+            rP = _rel(np.exp(view["tree_logP"][b, 1:n]), np.exp(tree.logP[1:n]))
+            rC = _rel(view["tree_C"][b, 1:n], tree.C[1:n])
+            rep.max_rel_p = max(rep.max_rel_p, rP); rep.max_rel_C = max(rep.max_rel_C, rC)
+            assert rP <= rtol and rC <= rtol
+    rep.near_tie_sequences = sum(near.values())
+    rep.diverged_sequences = sum(diverged.values())
+    rep.status_bits = bits
+    if own:
+        ctx.close()
+    return rep

