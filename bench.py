@@ -335,13 +335,48 @@ def run_cuda(args) -> None:
         dist.destroy_process_group()
 
 
+def run_profile(args) -> None:
+    """Levels 0 and 1 of the workload (64 + 640 logits rows) and the tail of the step, `steps` times."""
+    import paper_2502_13652_b200 as c2t
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = WORKLOAD
+    B, V, D, K, F, N = w["B"], w["V"], w["D"], w["K"], w["F"], w["N"]
+    w1, b1, w2, b2 = make_weights(w["hidden"])
+    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.BF16, max_depth=D, topk=K, frontier_cap=F, budget=N,
+                     threshold=w["beta"], hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2)
+    ctx = c2t.Context(cfg)
+    draft = [c2t_inputs.draft_logits(B, F, V, 0, l, torch.bfloat16, device=dev) for l in range(2)]
+    target = c2t_inputs.target_logits(B, ctx.Nw, V, 0, torch.bfloat16, device=dev)
+    root = c2t_inputs.root_tokens(B, V, 0).to(dev)
+    prefix = c2t_inputs.prefix_lengths(B).to(dev)
+    for _ in range(args.warmup + args.steps):
+        ctx.c2t_begin_step(root, prefix)
+        for l in range(2):
+            ctx.c2t_expand_level(l, draft[l])
+            ctx.c2t_prune(l)
+        ctx.c2t_prune(c2t.FINAL)
+        ctx.c2t_build_verify()
+        ctx.c2t_accept(target)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile": True, "launches": ctx.c2t_launch_count(),
+                      "n_nodes_mean": float(ctx.verify["n_nodes"].float().mean())}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--profile", action="store_true",
+                    help="small run for profiler captures: levels 0-1 of the workload plus rerank, verify "
+                         "inputs and accept; no end-to-end leg, no CPU baseline")
     args = ap.parse_args()
+    if args.profile:
+        args.steps = args.steps or 1
+        run_profile(args)
+        return
     if args.impl == "reference":
         args.steps = args.steps or 5
         run_reference(args)
