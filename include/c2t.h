@@ -187,6 +187,41 @@ typedef struct {
 int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride,
                int64_t row_stride, const c2t_accept_out *out, void *stream);
 
+/*
+ * The paper has no counterpart to this call; it exists for callers that cannot allocate.
+ *
+ * Some users of this library may not call cudaMalloc, and may not ask an allocator for a
+ * workspace either: an inference server that sized all of its device memory at start-up, a
+ * plug-in that runs inside someone else's engine, a latency-critical loop in which an
+ * allocation (which can synchronise the whole device) is forbidden.  For them this entry
+ * point computes the greedy token of every row of a logits matrix - the arg-max pass that
+ * c2t_accept runs over the target logits, ties to the lower token id, NaN ignored - without a
+ * context and without a workspace: the scratch memory it needs between its kernels is a fixed
+ * array that lives inside the library's device code.
+ *
+ *   logits_dev   [rows, vocab] of `dtype` (c2t_dtype), element offset of (r, v) = r*row_stride + v;
+ *                base 16-byte aligned, row_stride a multiple of 16 bytes
+ *   argmax_dev   [rows] int32, caller-owned; -1 for a row that holds only NaN
+ *
+ * Limits and rules:
+ *   - rows <= C2T_STATIC_MAX_ROWS and vocab <= C2T_STATIC_MAX_VOCAB; larger sizes are refused
+ *     with C2T_ERANGE.  The array takes about 2.1 MB on every GPU that loads the library,
+ *     until the process ends;
+ *   - the first call on a device looks the array's device address up (cudaGetSymbolAddress,
+ *     with that device current) and reads the SM count; make that first call once at start-up,
+ *     before any stream capture begins;
+ *   - the call only enqueues kernels on `stream`; it never calls cudaMalloc, cudaFree or any
+ *     allocating routine.  Work is done on the device that is current when it is called;
+ *   - all calls on a device share the one array and it keeps the last call's contents (the
+ *     call clears what it is about to use): two calls whose kernels can overlap on the GPU -
+ *     different streams, or different host threads without ordering - race on it.  Issue them
+ *     on one stream, or order them with events.
+ */
+#define C2T_STATIC_MAX_ROWS  4096
+#define C2T_STATIC_MAX_VOCAB 262144
+int c2t_row_argmax_static(const void *logits_dev, int32_t rows, int32_t vocab, int32_t dtype,
+                          int64_t row_stride, int32_t *argmax_dev, void *stream);
+
 /* Waits for `stream`, then ORs all sequences' status words into *bits_host and, if
  * per_seq_host is not NULL, copies the B words there.  For tests and debugging. */
 int c2t_status(c2t_ctx *ctx, uint32_t *bits_host, uint32_t *per_seq_host, void *stream);

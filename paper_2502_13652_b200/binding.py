@@ -114,6 +114,9 @@ def lib() -> C.CDLL:
         L.c2t_decode_step_host.argtypes = [C.c_void_p, P(c2t_host_step), C.c_void_p]
         L.c2t_launch_count.restype = C.c_int64
         L.c2t_launch_count.argtypes = [C.c_void_p]
+        L.c2t_row_argmax_static.restype = C.c_int
+        L.c2t_row_argmax_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                            C.c_void_p]
         L.c2t_strerror.restype = C.c_char_p
         L.c2t_strerror.argtypes = [C.c_int]
         _lib = L
@@ -194,6 +197,24 @@ def c2t_final_width(cfg: Config) -> int:
 def c2t_mask_words(cfg: Config) -> int:
     s, _keep = cfg.c_struct()
     return lib().c2t_mask_words(C.byref(s))
+
+
+STATIC_MAX_ROWS, STATIC_MAX_VOCAB = 4096, 262144
+
+
+def c2t_row_argmax_static(logits: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """Greedy token of every row of `logits` [rows, V] into `out` [rows] int32, using the scratch
+    array built into the library instead of a workspace: nothing is allocated by this call, which
+    is what a caller that may not allocate device memory needs.  Calls share that array, so keep
+    them on one stream (or order them); the first call on a device should precede any capture."""
+    assert logits.is_cuda and out.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
+    assert out.dtype == torch.int32 and out.is_contiguous() and out.numel() == logits.shape[0]
+    dtype = BF16 if logits.dtype == torch.bfloat16 else F32
+    assert logits.dtype in (torch.bfloat16, torch.float32)
+    with torch.cuda.device(logits.device):
+        _check(lib().c2t_row_argmax_static(logits.data_ptr(), logits.shape[0], logits.shape[1], dtype,
+                                           logits.stride(0), out.data_ptr(), _stream(stream)),
+               "c2t_row_argmax_static")
 
 
 class Context:
