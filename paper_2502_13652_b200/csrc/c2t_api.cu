@@ -113,6 +113,7 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   s.info_target = w.take<PassInfo>(1);
   s.part_stats = w.take<float4>(B * F * ms);
   s.part_keys = w.take<unsigned long long>(B * F * ms * K);
+  s.part_held = w.take<unsigned long long>(B * F * ms * kHeldPerSlot);
   s.part_best = w.take<unsigned long long>(B * Nw * ms);
   s.w1 = w.take<float>(3 * C2T_MAX_HIDDEN);
   s.b1 = w.take<float>(C2T_MAX_HIDDEN);
@@ -231,7 +232,7 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   p.counts = t.frontier_n[level & 1];
   p.max_splits = t.max_splits;
   p.info = t.info_draft;
-  p.part_stats = t.part_stats; p.part_keys = t.part_keys;
+  p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
   if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid, (cudaStream_t)stream) != cudaSuccess)
     return C2T_ECUDA;
   ctx->launches += 1;

@@ -28,15 +28,16 @@ __device__ __forceinline__ int32_t key_token(unsigned long long k) {
   return (int32_t)(0xFFFFFFFFu - (uint32_t)k);
 }
 
-// Logits of -inf are read as the lowest finite value of the storage type, so that
-// "probability zero" never produces inf - inf or 0 * inf in the running sums.
-constexpr float kNegInfAsFinite = -3.38e38f;   // anything at or below this was -inf (or as good as)
+// Logits of -inf (and anything below -2^127) are read as -2^127, so that "probability zero"
+// never produces inf - inf or 0 * inf in the running sums.
+constexpr float kNegInfAsFinite = -1.7e38f;   // anything at or below this was -inf (or as good as)
 
 // ---------------------------------------------------------------- vocab pass -
 
 constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass
 constexpr int kPassCtasPerSm = 2;
 constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors than this
+constexpr int kHeldPerSlot = kPassThreads / 32;   // exact keys held out of the fp32 sums, one per warp
 
 // What one launch of the vocabulary pass derived from the device-side row counts.
 struct PassInfo {
@@ -54,8 +55,9 @@ struct PassParams {
   int32_t max_splits;               // partial slots per row
   PassInfo *info;                   // written by CTA 0
   // expand: per (row, split) partial
-  float4 *part_stats;               // {m_ref, S, T, n_keys as int bits}
-  unsigned long long *part_keys;    // [.. * K] sorted descending, 0-padded
+  float4 *part_stats;               // {offset c, S, U, n_keys as int bits}: base-2 sums, see expand_pass.cu
+  unsigned long long *part_keys;    // [.. * K] the segment's K largest keys, sorted descending, 0-padded
+  unsigned long long *part_held;    // [.. * kHeldPerSlot] keys excluded from S and U (0 = none)
   // argmax: per (row, split) best key
   unsigned long long *part_best;
 };
@@ -91,6 +93,7 @@ struct TreeState {
   PassInfo *info_draft, *info_target;
   float4 *part_stats;
   unsigned long long *part_keys;
+  unsigned long long *part_held;
   unsigned long long *part_best;
   float *w1, *b1, *w2, *b2;
 };

@@ -134,10 +134,11 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     const size_t slot0 = (size_t)a * t.max_splits;
     const int n_keys = n_splits * K;
 
-    // the row maximum is the largest key of any partial
+    // the row maximum is the largest key held out of any partial's sums
+    const int n_held = n_splits * kHeldPerSlot;
     unsigned long long top = 0ull;
-    for (int i = lane; i < n_splits; i += 32) {
-      unsigned long long k0 = t.part_keys[(slot0 + i) * K];
+    for (int i = lane; i < n_held; i += 32) {
+      unsigned long long k0 = t.part_held[slot0 * kHeldPerSlot + i];
       top = k0 > top ? k0 : top;
     }
 #pragma unroll
@@ -147,19 +148,33 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     }
     const double M = (double)key_value(top);
 
-    // fp32 tails of every split, rescaled to M
+    // fp32 sums of every split: S = sum 2^t, U = sum 2^t t with t = x log2(e) + c, brought to
+    // natural units relative to M:  x - M = t ln2 + g,  g = -c ln2 - M
     double S = 0.0, T = 0.0;
     for (int i = lane; i < n_splits; i += 32) {
       float4 st = t.part_stats[slot0 + i];
-      double Ss = (double)st.y, Ts = (double)st.z;
-      if (Ss != 0.0 || Ts != 0.0) {               // (NaN passes this test and poisons the sums)
-        double d = (double)st.x - M;
-        double f = exp(d);
+      const double Ss = (double)st.y, Us = (double)st.z;
+      if (Ss != 0.0 || Us != 0.0) {               // (NaN passes this test and poisons the sums)
+        const double kLn2 = 0.69314718055994530942;
+        const double g = -(double)st.x * kLn2 - M;
+        const double f = exp(g);
         S += Ss * f;
-        T += f * (Ts + d * Ss);
+        T += f * (kLn2 * Us + g * Ss);
       }
     }
-    // exact keys: rank them; all but the row maximum join the sums; the K best become candidates
+    // held-out elements are not in those sums: add them exactly, all but the row maximum itself
+    for (int i = lane; i < n_held; i += 32) {
+      const unsigned long long key = t.part_held[slot0 * kHeldPerSlot + i];
+      if (key == 0ull || key == top) continue;
+      const float x = key_value(key);
+      if (x > kNegInfAsFinite) {
+        double d = (double)x - M;
+        double e = exp(d);
+        S += e;
+        T += e * d;
+      }
+    }
+    // the K best keys over all splits become the candidates
     for (int i = lane; i < n_keys; i += 32) {
       const unsigned long long key = t.part_keys[slot0 * K + i];
       if (key == 0ull) continue;
@@ -170,14 +185,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
         unsigned long long other = t.part_keys[slot0 * K + r];
         rank += (other > key) && (key_token(other) < t.V);
       }
-      const float x = key_value(key);
-      if (key != top && x > kNegInfAsFinite) {
-        double d = (double)x - M;
-        double e = exp(d);
-        S += e;
-        T += e * d;
-      }
-      if (rank < K) { s_x[j * K + rank] = x; s_tok[j * K + rank] = tok; }
+      if (rank < K) { s_x[j * K + rank] = key_value(key); s_tok[j * K + rank] = tok; }
     }
     S = warp_sum(S);
     T = warp_sum(T);

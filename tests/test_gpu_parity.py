@@ -183,7 +183,10 @@ def test_special_rows(kind, dtype):
     root = torch.zeros(B, dtype=torch.int32); prefix = torch.full((B,), 9, dtype=torch.int32)
     rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
     print(f"\n  [{kind} {dtype}] {rep.line()}")
-    assert rep.status_bits == 0 and rep.diverged_sequences == 0
+    assert rep.status_bits == 0
+    # all-equal rows tie every candidate exactly in the oracle; the CUDA path's fp32 tail sums depend on
+    # where a row is cut into segments, so there the tie is broken by rounding (a counted near tie)
+    assert rep.diverged_sequences == 0 or (kind == "uniform" and rep.diverged_sequences <= rep.near_tie_sequences)
     if kind == "uniform":
         ctx = c2t.Context(gcfg)
         ctx.c2t_begin_step(root.cuda(), prefix.cuda())
