@@ -168,7 +168,7 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   if (workspace_bytes < carve(cfg, nullptr, nullptr)) return C2T_ERANGE;
   if (cudaSetDevice(cfg->device) != cudaSuccess) { cudaGetLastError(); return C2T_ECUDA; }
   const int grid = pass_grid(cfg->device);
-  if (grid < 0) { cudaGetLastError(); return C2T_ECUDA; }
+  if (grid < 0 || prepare_expand_pass() != cudaSuccess) { cudaGetLastError(); return C2T_ECUDA; }
 
   c2t_ctx *ctx = new (std::nothrow) c2t_ctx;
   if (!ctx) return C2T_EINVAL;

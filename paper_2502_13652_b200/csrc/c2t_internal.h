@@ -64,6 +64,7 @@ struct PassParams {
 
 int max_splits_for(int vocab, int elem_bytes, int grid);
 
+cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
 cudaError_t launch_argmax_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
 

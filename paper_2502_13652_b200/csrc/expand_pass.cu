@@ -9,10 +9,12 @@
 // head of another; each (row, CTA) piece is a "segment" and produces one partial record.  The
 // pruning kernel merges the partials of a row in double precision.
 //
-// Data movement.  A thread reads groups of four 16-byte vectors, 512 vectors apart, with plain
-// 128-bit loads issued back to back.  The first group of the next segment is requested before
-// the closing barriers of the current one.  Nothing waits on another thread's progress except
-// at __syncthreads.
+// Data movement.  A thread works on groups of four 16-byte vectors, 512 vectors apart.  Each
+// thread owns 4 x 16 bytes in each of two shared-memory slots and fills them with cp.async:
+// while group n is in registers, groups n+1 and n+2 are in flight, across segment boundaries
+// too.  A thread reads back only what it copied itself, so the only wait is on its own copies
+// (cp.async.wait_group); nothing waits on another thread's progress except at __syncthreads,
+// of which a segment boundary has two.
 //
 // Sums.  In base-2 units relative to a warp-uniform offset c = -m log2(e):  t = x log2(e) + c,
 // S = sum 2^t, U = sum 2^t t  (one unpack, FMA, ex2, add, FMA per element).  They cover all
@@ -252,28 +254,77 @@ struct SegWalk {
   }
 };
 
-// Issues the loads of a thread's group (vectors vt, vt+NT, vt+2NT, vt+3NT of a segment ending
-// at v1).  In the common case (all four are whole vectors inside the segment, for every lane)
-// the four loads go out back to back with nothing between them; vectors past the segment end
-// are filled with -2^127.
-template <bool BF16>
-__device__ __forceinline__ void load_group(Group &g, const char *row, int vt, int v1, int v_full, int V) {
-  using VT = Vec<BF16>;
-  const int lim = v1 < v_full ? v1 : v_full;
-  if (__all_sync(kFull, vt + 3 * NT < lim)) {
-    const uint4 *base = reinterpret_cast<const uint4 *>(row) + vt;
-    g.q[0] = ldg_stream(base);
-    g.q[1] = ldg_stream(base + NT);
-    g.q[2] = ldg_stream(base + 2 * NT);
-    g.q[3] = ldg_stream(base + 3 * NT);
-  } else {
-    const uint32_t lo = BF16 ? kLowestBf16x2 : __float_as_uint(kLowestF32);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      g.q[u] = make_uint4(lo, lo, lo, lo);
-      if (vt + u * NT < v1) g.q[u] = VT::load(row, vt + u * NT, v_full, V);
+// ---------------------------------------------------------------- asynchronous prefetch ring
+//
+// Every thread owns 4 x 16 bytes in each of the two slots of a shared-memory ring and fills
+// them with cp.async (global -> shared, no registers held): while group n is being worked on,
+// groups n+1 and n+2 are in flight.  A thread only ever reads back what it copied itself, so
+// the only wait is cp.async.wait_group on its own copies; no barrier is involved and the
+// prefetch runs ahead across segment boundaries.
+
+__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gmem_src) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// The groups of a span in order: group = four vectors per thread, NT apart, of one segment.
+struct GroupCursor {
+  SegWalk walk;
+  Segment seg;     // the segment the current group belongs to
+  int tv0;         // first vector of the current group (CTA-uniform); the thread's are tv0+tid+u*NT
+  bool valid;
+  __device__ GroupCursor(const Partition &pt, const PassParams &p, const int *s_off, size_t esz) : walk(pt) {
+    seg = walk.take(p, s_off, esz);
+    tv0 = seg.v0;
+    valid = true;
+  }
+  __device__ bool last_of_segment() const { return tv0 + 4 * NT >= seg.v1; }
+  __device__ void advance(const PassParams &p, const int *s_off, size_t esz) {
+    tv0 += 4 * NT;
+    if (tv0 >= seg.v1) {
+      if (walk.done()) { valid = false; return; }
+      seg = walk.take(p, s_off, esz);
+      tv0 = seg.v0;
     }
   }
+};
+
+// Requests the whole vectors of the cursor's group into the thread's places of a ring slot.
+__device__ __forceinline__ void prefetch_group(const GroupCursor &c, uint4 *slot, int v_full) {
+  if (c.valid) {
+    const int lim = c.seg.v1 < v_full ? c.seg.v1 : v_full;
+    const uint4 *src = reinterpret_cast<const uint4 *>(c.seg.row) + c.tv0 + (int)threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (c.tv0 + (int)threadIdx.x + u * NT < lim) cp_async_16(slot + threadIdx.x + u * NT, src + u * NT);
+  }
+  cp_async_commit();
+}
+
+// Takes the cursor's group out of a ring slot (its copies have completed) into registers and
+// clamps it.  Vectors past the segment end become -2^127, which adds exactly 0 to the sums; a
+// ragged last vector of a row is assembled from scalar loads.
+template <bool BF16>
+__device__ __forceinline__ void take_group(Group &g, const GroupCursor &c, const uint4 *slot, int v_full, int V) {
+  using VT = Vec<BF16>;
+  const uint32_t lo = BF16 ? kLowestBf16x2 : __float_as_uint(kLowestF32);
+  const int vt = c.tv0 + (int)threadIdx.x;
+  if (__all_sync(kFull, vt + 3 * NT < (c.seg.v1 < v_full ? c.seg.v1 : v_full))) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) g.q[u] = slot[threadIdx.x + u * NT];
+  } else {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = vt + u * NT;
+      g.q[u] = make_uint4(lo, lo, lo, lo);
+      if (v < c.seg.v1) g.q[u] = v < v_full ? slot[threadIdx.x + u * NT] : VT::load(c.seg.row, v, v_full, V);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u) VT::clamp(g.q[u]);
 }
 
 // Exact fallback for a segment whose candidate buffer overflowed: K rounds of a CTA-wide
@@ -313,10 +364,10 @@ __device__ __noinline__ void select_by_rescan(int K, int V, int v_full, const ch
   }
 }
 
-// Start of a segment: the lane maxima of the first group seed the filter (K-th largest lane
-// maximum: a valid lower bound of the K-th largest element) and the reference (their maximum).
+// Warm-up, stage 1 (every warp, no barrier): the warp's K largest lane maxima of a segment's
+// first group, descending, into shared memory.
 template <bool BF16>
-__device__ __forceinline__ void segment_begin(SegShared &sh, int K, const Group &g, int vt, int v1, SegState &st) {
+__device__ __forceinline__ void warmup_stage1(SegShared &sh, int K, const Group &g, int vt, int v1) {
   using VT = Vec<BF16>;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float lmax = -INFINITY;
@@ -327,35 +378,39 @@ __device__ __forceinline__ void segment_begin(SegShared &sh, int K, const Group 
       if (vm == vm) lmax = fmaxf(lmax, vm);
     }
   }
-  {  // the warp's K largest lane maxima, descending, into shared memory
-    uint32_t live = f32_orderable(__float_as_uint(lmax)), mine = 0;
-    for (int r = 0; r < K; ++r) {
-      const uint32_t mx = __reduce_max_sync(kFull, live);
-      const unsigned bal = __ballot_sync(kFull, live == mx);
-      if (lane == __ffs(bal) - 1) live = 0;
-      if (lane == r) mine = mx;
-    }
-    if (lane < K) sh.warm[warp * K + lane] = mine;
+  uint32_t live = f32_orderable(__float_as_uint(lmax)), mine = 0;
+  for (int r = 0; r < K; ++r) {
+    const uint32_t mx = __reduce_max_sync(kFull, live);
+    const unsigned bal = __ballot_sync(kFull, live == mx);
+    if (lane == __ffs(bal) - 1) live = 0;
+    if (lane == r) mine = mx;
   }
-  __syncthreads();
-  if (warp == 0) {  // K-th largest of the union of the sorted per-warp lists: lane w walks list w
-    int head = 0;
-    uint32_t mx = 0, first = 0;
-    for (int r = 0; r < K; ++r) {
-      const uint32_t h = (lane < kWarps && head < K) ? sh.warm[lane * K + head] : 0u;
-      mx = __reduce_max_sync(kFull, h);
-      if (r == 0) first = mx;
-      const unsigned bal = __ballot_sync(kFull, h == mx);
-      if (lane == __ffs(bal) - 1) ++head;
-    }
-    if (lane < K) sh.vals[lane] = mx;
-    if (lane == 0) {
-      sh.m0 = __uint_as_float(f32_from_orderable(first));
-      sh.cnt = 0;
-      sh.overflow = 0;
-    }
+  if (lane < K) sh.warm[warp * K + lane] = mine;
+}
+
+// Warm-up, stage 2 (warp 0, between two barriers): the K-th largest of the union of the sorted
+// per-warp lists seeds the filter (a valid lower bound of the segment's K-th largest element),
+// their maximum becomes the reference of the sums; the candidate buffer is emptied.
+__device__ __forceinline__ void warmup_stage2(SegShared &sh, int K) {
+  const int lane = threadIdx.x & 31;
+  int head = 0;
+  uint32_t mx = 0, first = 0;
+  for (int r = 0; r < K; ++r) {   // lane w walks list w
+    const uint32_t h = (lane < kWarps && head < K) ? sh.warm[lane * K + head] : 0u;
+    mx = __reduce_max_sync(kFull, h);
+    if (r == 0) first = mx;
+    const unsigned bal = __ballot_sync(kFull, h == mx);
+    if (lane == __ffs(bal) - 1) ++head;
   }
-  __syncthreads();
+  if (lane < K) sh.vals[lane] = mx;
+  if (lane == 0) {
+    sh.m0 = __uint_as_float(f32_from_orderable(first));
+    sh.cnt = 0;
+    sh.overflow = 0;
+  }
+}
+
+__device__ __forceinline__ void state_init(const SegShared &sh, SegState &st) {
   acc_clear(st.acc);
   st.m = sh.m0;                                      // warp-uniform reference of the sums
   st.c = -st.m * kLog2e;
@@ -363,14 +418,9 @@ __device__ __forceinline__ void segment_begin(SegShared &sh, int K, const Group 
   st.held = 0ull;
 }
 
-// End of a segment: merge the sums in a fixed order and emit the partial record.
-template <bool BF16>
-__device__ __forceinline__ void segment_end(SegShared &sh, const PassParams &p, const Partition &pt,
-                                            const Segment &g, const SegState &st) {
+// End of a segment, every warp, before the barrier: the warp's sums (fixed order) and held key.
+__device__ __forceinline__ void publish_warp_sums(SegShared &sh, const SegState &st) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int K = p.K;
-  const int split = blockIdx.x - (int)(((long long)g.a * pt.vec_per_row) / pt.span);
-  const size_t slot = (size_t)g.a * p.max_splits + split;
   float S = st.acc.S0 + st.acc.S1, U = st.acc.U0 + st.acc.U1;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {                   // the offset is warp-uniform: plain sums
@@ -381,62 +431,86 @@ __device__ __forceinline__ void segment_end(SegShared &sh, const PassParams &p, 
     sh.red[warp][0] = st.c; sh.red[warp][1] = S; sh.red[warp][2] = U;
     sh.held[warp] = st.held;
   }
-  __syncthreads();
-  const bool overflow = sh.overflow != 0;
-  if (warp == 0) {
-    float cc = lane < kWarps ? sh.red[lane][0] : sh.red[0][0];
-    S = lane < kWarps ? sh.red[lane][1] : 0.f;
-    U = lane < kWarps ? sh.red[lane][2] : 0.f;
+}
+
+// End of a segment, warp 0, after the barrier: merge the warps' sums and emit the partial record.
+__device__ __forceinline__ void emit_partial(SegShared &sh, const PassParams &p, size_t slot, bool overflow) {
+  const int lane = threadIdx.x & 31;
+  const int K = p.K;
+  float cc = lane < kWarps ? sh.red[lane][0] : sh.red[0][0];
+  float S = lane < kWarps ? sh.red[lane][1] : 0.f;
+  float U = lane < kWarps ? sh.red[lane][2] : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float c_o = __shfl_down_sync(kFull, cc, o);
-      const float S_o = __shfl_down_sync(kFull, S, o);
-      const float U_o = __shfl_down_sync(kFull, U, o);
-      combine(cc, S, U, c_o, S_o, U_o);
-    }
-    if (lane < kWarps) p.part_held[slot * kWarps + lane] = sh.held[lane];
-    int n_keys = K;
-    if (!overflow) {
-      // the K largest keys of the buffer, sorted, by counting
-      const int n = sh.cnt < kBufCap ? sh.cnt : kBufCap;
-      n_keys = n < K ? n : K;
+  for (int o = 16; o > 0; o >>= 1) {
+    const float c_o = __shfl_down_sync(kFull, cc, o);
+    const float S_o = __shfl_down_sync(kFull, S, o);
+    const float U_o = __shfl_down_sync(kFull, U, o);
+    combine(cc, S, U, c_o, S_o, U_o);
+  }
+  if (lane < kWarps) p.part_held[slot * kWarps + lane] = sh.held[lane];
+  int n_keys = K;
+  if (!overflow) {
+    // the K largest keys of the buffer, sorted, by counting
+    const int n = sh.cnt < kBufCap ? sh.cnt : kBufCap;
+    n_keys = n < K ? n : K;
+    if (n <= 32) {                                      // one key per lane, ranked through shuffles
+      const unsigned long long key = lane < n ? sh.buf[lane] : 0ull;
+      int rank = 0;
+      for (int r = 0; r < n; ++r) rank += __shfl_sync(kFull, key, r) > key;
+      if (lane < n && rank < K) p.part_keys[slot * K + rank] = key;
+    } else {
       for (int i = lane; i < n; i += 32) {
         const unsigned long long key = sh.buf[i];
         int rank = 0;
         for (int r = 0; r < n; ++r) rank += sh.buf[r] > key;
         if (rank < K) p.part_keys[slot * K + rank] = key;
       }
-      for (int r = n_keys + lane; r < K; r += 32) p.part_keys[slot * K + r] = 0ull;
     }
-    if (lane == 0) p.part_stats[slot] = make_float4(cc, S, U, __int_as_float(n_keys));
+    for (int r = n_keys + lane; r < K; r += 32) p.part_keys[slot * K + r] = 0ull;
   }
-  if (overflow) select_by_rescan<BF16>(K, p.V, pt.v_full, g.row, g.v0, g.v1, p.part_keys + slot * K, sh.held);
-  __syncthreads();
+  if (lane == 0) p.part_stats[slot] = make_float4(cc, S, U, __int_as_float(n_keys));
 }
 
 template <bool BF16>
 __global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) expand_pass_kernel(PassParams p) {
   using VT = Vec<BF16>;
-  __shared__ int s_off[C2T_MAX_BATCH + 1];
+  extern __shared__ __align__(16) unsigned char s_dyn[];     // ring: 2 slots of 4*NT vectors, then row offsets
   __shared__ SegShared sh;
+  uint4 *ring = reinterpret_cast<uint4 *>(s_dyn);
+  int *s_off = reinterpret_cast<int *>(s_dyn + 2 * 4 * NT * sizeof(uint4));
 
   const int K = p.K;
+  const int warp = threadIdx.x >> 5;
   const int n_rows = build_row_offsets(p.counts, p.B, p.rows_per_seq_max, s_off);
   const Partition pt = make_partition<VT::N>(p, n_rows);
   if (pt.start >= pt.end) return;
 
   const size_t esz = BF16 ? 2 : 4;
-  SegWalk walk(pt);
-  Segment seg = walk.take(p, s_off, esz);
+  GroupCursor cur(pt, p, s_off, esz);      // the group being worked on
+  GroupCursor pre = cur;                   // the group being requested, two ahead
+  prefetch_group(pre, ring, pt.v_full);
+  pre.advance(p, s_off, esz);
+  prefetch_group(pre, ring + 4 * NT, pt.v_full);
+  pre.advance(p, s_off, esz);
+  unsigned n = 0;                          // index of the current group: its ring slot is n & 1
+
   Group g;
-  load_group<BF16>(g, seg.row, seg.v0 + (int)threadIdx.x, seg.v1, pt.v_full, p.V);
+  cp_async_wait<1>();
+  take_group<BF16>(g, cur, ring, pt.v_full, p.V);
+  prefetch_group(pre, ring, pt.v_full);
+  pre.advance(p, s_off, esz);
+  warmup_stage1<BF16>(sh, K, g, cur.tv0 + (int)threadIdx.x, cur.seg.v1);
+  __syncthreads();
+  if (warp == 0) warmup_stage2(sh, K);
+  __syncthreads();
+
   for (;;) {
+    // ---- one segment; its first group is in registers and the filter is seeded
+    const Segment seg = cur.seg;
     SegState st;
-    int vt = seg.v0 + (int)threadIdx.x;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) VT::clamp(g.q[u]);
-    segment_begin<BF16>(sh, K, g, vt, seg.v1, st);
+    state_init(sh, st);
     for (;;) {
+      const int vt = cur.tv0 + (int)threadIdx.x;
       st.thr = __uint_as_float(f32_from_orderable(*reinterpret_cast<volatile uint32_t *>(&sh.vals[K - 1])));
       const float vm4 = fmaxf(fmaxf(VT::vmax(g.q[0]), VT::vmax(g.q[1])), fmaxf(VT::vmax(g.q[2]), VT::vmax(g.q[3])));
       if (__any_sync(kFull, vm4 > st.mw && vt < seg.v1)) {
@@ -446,23 +520,34 @@ __global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) expand_pass_kern
 #pragma unroll
         for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], st.c);
       }
-      vt += 4 * NT;
-      if (vt - (int)threadIdx.x >= seg.v1) break;          // CTA-uniform: the group's first vector
-      load_group<BF16>(g, seg.row, vt, seg.v1, pt.v_full, p.V);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) VT::clamp(g.q[u]);
+      const bool last = cur.last_of_segment();
+      cur.advance(p, s_off, esz);
+      ++n;
+      if (cur.valid) {                       // next group (of this or of the next segment) into registers
+        cp_async_wait<1>();
+        uint4 *slot = ring + (n & 1u) * 4 * NT;
+        take_group<BF16>(g, cur, slot, pt.v_full, p.V);
+        prefetch_group(pre, slot, pt.v_full);
+        pre.advance(p, s_off, esz);
+      }
+      if (last) break;
     }
-    // the first group of the next segment is requested before this segment's closing barriers
-    const bool more = !walk.done();
-    Segment next = seg;
-    if (more) {
-      next = walk.take(p, s_off, esz);
-      load_group<BF16>(g, next.row, next.v0 + (int)threadIdx.x, next.v1, pt.v_full, p.V);
-    }
-    segment_end<BF16>(sh, p, pt, seg, st);
+    // ---- segment boundary: two barriers; warp 0 closes this segment and seeds the next
+    publish_warp_sums(sh, st);
+    const bool more = cur.valid;
+    if (more) warmup_stage1<BF16>(sh, K, g, cur.tv0 + (int)threadIdx.x, cur.seg.v1);
+    __syncthreads();
+    const bool overflow = sh.overflow != 0;
+    const int split = blockIdx.x - (int)(((long long)seg.a * pt.vec_per_row) / pt.span);
+    const size_t slot_id = (size_t)seg.a * p.max_splits + split;
+    if (warp == 0) emit_partial(sh, p, slot_id, overflow);
+    if (overflow)
+      select_by_rescan<BF16>(K, p.V, pt.v_full, seg.row, seg.v0, seg.v1, p.part_keys + slot_id * K, sh.held);
+    if (warp == 0 && more) warmup_stage2(sh, K);
+    __syncthreads();
     if (!more) break;
-    seg = next;
   }
+  cp_async_wait<0>();
 }
 
 }  // namespace
@@ -475,9 +560,21 @@ int max_splits_for(int vocab, int elem_bytes, int grid) {
   return by_span + 1;
 }
 
+static size_t expand_dynamic_smem(int B) {
+  return 2 * 4 * (size_t)kPassThreads * sizeof(uint4) + ((size_t)B + 1) * sizeof(int);
+}
+
+cudaError_t prepare_expand_pass() {
+  const int bytes = (int)expand_dynamic_smem(C2T_MAX_BATCH);
+  cudaError_t e = cudaFuncSetAttribute(expand_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(expand_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s) {
-  if (dtype == C2T_BF16) expand_pass_kernel<true><<<grid, kPassThreads, 0, s>>>(p);
-  else expand_pass_kernel<false><<<grid, kPassThreads, 0, s>>>(p);
+  const size_t smem = expand_dynamic_smem(p.B);
+  if (dtype == C2T_BF16) expand_pass_kernel<true><<<grid, kPassThreads, smem, s>>>(p);
+  else expand_pass_kernel<false><<<grid, kPassThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 
