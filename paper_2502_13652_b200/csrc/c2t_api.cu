@@ -9,7 +9,8 @@ using namespace c2t;
 struct c2t_ctx {
   c2t_config cfg;
   TreeState t;
-  int grid;              // CTAs of the vocabulary pass
+  int grid;              // CTAs of the arg-max pass
+  int grid_expand;       // CTAs of the expand pass
   int next_level;        // level the next c2t_expand_level must carry
   int expanded;          // 1 after expand_level(next_level), before its prune
   int finalized;         // 1 after c2t_prune(C2T_FINAL)
@@ -78,7 +79,7 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   const size_t B = c->batch, F = c->frontier_cap, K = c->topk;
   const size_t cap = tree_capacity_unchecked(c), Nw = c2t_final_width(c);
   const int eb = c->dtype == C2T_BF16 ? 2 : 4;
-  const size_t ms = max_splits_for(c->vocab, eb, kMaxSms * kPassCtasPerSm);
+  const size_t ms = max_splits_for(c->vocab, eb, kMaxSms * (kExpandCtasPerSm > kPassCtasPerSm ? kExpandCtasPerSm : kPassCtasPerSm));
   TreeState s;
   memset(&s, 0, sizeof s);
   for (int i = 0; i < 2; ++i) {
@@ -176,6 +177,7 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   ctx->cfg = *cfg;
   ctx->cfg.w1 = ctx->cfg.b1 = ctx->cfg.w2 = ctx->cfg.b2 = nullptr;
   ctx->grid = grid;
+  ctx->grid_expand = grid / kPassCtasPerSm * kExpandCtasPerSm;
   ctx->elem_bytes = cfg->dtype == C2T_BF16 ? 2 : 4;
   carve(cfg, workspace_dev, &ctx->t);
   TreeState &t = ctx->t;
@@ -184,8 +186,8 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   t.cap = tree_capacity_unchecked(cfg);
   t.hidden = cfg->classifier == C2T_CLS_MLP ? cfg->hidden : 0;
   t.classifier = cfg->classifier; t.tree_add = cfg->tree_add; t.beta = cfg->threshold;
-  t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, grid);
-  t.max_splits_tgt = t.max_splits;
+  t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid_expand);
+  t.max_splits_tgt = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid);
 
   cudaError_t e = cudaSuccess;
   if (cfg->classifier == C2T_CLS_MLP) {
@@ -233,7 +235,7 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   p.max_splits = t.max_splits;
   p.info = t.info_draft;
   p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
-  if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid, (cudaStream_t)stream) != cudaSuccess)
+  if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid_expand, (cudaStream_t)stream) != cudaSuccess)
     return C2T_ECUDA;
   ctx->launches += 1;
   ctx->expanded = 1;

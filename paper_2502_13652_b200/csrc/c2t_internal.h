@@ -37,7 +37,11 @@ constexpr float kNegInfAsFinite = -1.7e38f;   // anything at or below this was -
 constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass
 constexpr int kPassCtasPerSm = 2;
 constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors than this
-constexpr int kHeldPerSlot = kPassThreads / 32;   // exact keys held out of the fp32 sums, one per warp
+// the expand pass runs more, smaller CTAs: no register spills at 80 registers per thread, and
+// while one CTA is at a segment boundary the others on the SM keep streaming
+constexpr int kExpandThreads = 256;
+constexpr int kExpandCtasPerSm = 3;
+constexpr int kHeldPerSlot = kExpandThreads / 32;   // exact keys held out of the fp32 sums, one per warp
 
 // What one launch of the vocabulary pass derived from the device-side row counts.
 struct PassInfo {

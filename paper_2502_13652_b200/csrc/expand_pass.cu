@@ -4,12 +4,12 @@
 //
 // Work partition.  The active rows (a device-side count per sequence) are laid end to end as
 // n_rows * vec_per_row 16-byte vectors and cut into equal contiguous spans, one per CTA of a
-// persistent grid (two CTAs of 512 threads per SM), so every CTA streams the same number of
+// persistent grid (three CTAs of 256 threads per SM), so every CTA streams the same number of
 // bytes whatever the row count.  A span may cover the tail of one row, some whole rows and the
 // head of another; each (row, CTA) piece is a "segment" and produces one partial record.  The
 // pruning kernel merges the partials of a row in double precision.
 //
-// Data movement.  A thread works on groups of four 16-byte vectors, 512 vectors apart.  Each
+// Data movement.  A thread works on groups of four 16-byte vectors, 256 vectors apart.  Each
 // thread owns 4 x 16 bytes in each of two shared-memory slots and fills them with cp.async:
 // while group n is in registers, groups n+1 and n+2 are in flight, across segment boundaries
 // too.  A thread reads back only what it copied itself, so the only wait is on its own copies
@@ -42,7 +42,8 @@
 namespace c2t {
 namespace {
 
-constexpr int NT = kPassThreads;   // 512
+constexpr int NT = kExpandThreads;
+constexpr int kEWarps = NT / 32;
 constexpr int kBufCap = 256;       // top-K candidate keys a segment can collect before the exact fallback
 
 // ---------------------------------------------------------------- sums
@@ -117,10 +118,10 @@ __device__ __forceinline__ void mask_element(uint4 &q, int i) {
 // Shared by the CTA for the segment being streamed.
 struct SegShared {
   unsigned long long buf[kBufCap];        // keys of every element that met the filter when it was read
-  unsigned long long held[kWarps];        // per warp: the key held out of the sums
+  unsigned long long held[kEWarps];        // per warp: the key held out of the sums
   uint32_t vals[C2T_MAX_TOPK];            // K largest values seen (orderable form); vals[K-1] is the filter
-  uint32_t warm[kWarps * C2T_MAX_TOPK];
-  float red[kWarps][3];
+  uint32_t warm[kEWarps * C2T_MAX_TOPK];
+  float red[kEWarps][3];
   float m0;
   int cnt;
   int overflow;
@@ -358,7 +359,7 @@ __device__ __noinline__ void select_by_rescan(int K, int V, int v_full, const ch
     if (lane == 0) s_scratch[warp] = best;
     __syncthreads();
     best = 0ull;
-    for (int w = 0; w < kWarps; ++w) best = s_scratch[w] > best ? s_scratch[w] : best;
+    for (int w = 0; w < kEWarps; ++w) best = s_scratch[w] > best ? s_scratch[w] : best;
     if (tid == 0) out_keys[r] = best;
     bound = best;
   }
@@ -396,7 +397,7 @@ __device__ __forceinline__ void warmup_stage2(SegShared &sh, int K) {
   int head = 0;
   uint32_t mx = 0, first = 0;
   for (int r = 0; r < K; ++r) {   // lane w walks list w
-    const uint32_t h = (lane < kWarps && head < K) ? sh.warm[lane * K + head] : 0u;
+    const uint32_t h = (lane < kEWarps && head < K) ? sh.warm[lane * K + head] : 0u;
     mx = __reduce_max_sync(kFull, h);
     if (r == 0) first = mx;
     const unsigned bal = __ballot_sync(kFull, h == mx);
@@ -437,9 +438,9 @@ __device__ __forceinline__ void publish_warp_sums(SegShared &sh, const SegState 
 __device__ __forceinline__ void emit_partial(SegShared &sh, const PassParams &p, size_t slot, bool overflow) {
   const int lane = threadIdx.x & 31;
   const int K = p.K;
-  float cc = lane < kWarps ? sh.red[lane][0] : sh.red[0][0];
-  float S = lane < kWarps ? sh.red[lane][1] : 0.f;
-  float U = lane < kWarps ? sh.red[lane][2] : 0.f;
+  float cc = lane < kEWarps ? sh.red[lane][0] : sh.red[0][0];
+  float S = lane < kEWarps ? sh.red[lane][1] : 0.f;
+  float U = lane < kEWarps ? sh.red[lane][2] : 0.f;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float c_o = __shfl_down_sync(kFull, cc, o);
@@ -447,7 +448,7 @@ __device__ __forceinline__ void emit_partial(SegShared &sh, const PassParams &p,
     const float U_o = __shfl_down_sync(kFull, U, o);
     combine(cc, S, U, c_o, S_o, U_o);
   }
-  if (lane < kWarps) p.part_held[slot * kWarps + lane] = sh.held[lane];
+  if (lane < kEWarps) p.part_held[slot * kEWarps + lane] = sh.held[lane];
   int n_keys = K;
   if (!overflow) {
     // the K largest keys of the buffer, sorted, by counting
@@ -472,7 +473,7 @@ __device__ __forceinline__ void emit_partial(SegShared &sh, const PassParams &p,
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) expand_pass_kernel(PassParams p) {
+__global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_kernel(PassParams p) {
   using VT = Vec<BF16>;
   extern __shared__ __align__(16) unsigned char s_dyn[];     // ring: 2 slots of 4*NT vectors, then row offsets
   __shared__ SegShared sh;
@@ -561,7 +562,7 @@ int max_splits_for(int vocab, int elem_bytes, int grid) {
 }
 
 static size_t expand_dynamic_smem(int B) {
-  return 2 * 4 * (size_t)kPassThreads * sizeof(uint4) + ((size_t)B + 1) * sizeof(int);
+  return 2 * 4 * (size_t)kExpandThreads * sizeof(uint4) + ((size_t)B + 1) * sizeof(int);
 }
 
 cudaError_t prepare_expand_pass() {
@@ -573,8 +574,8 @@ cudaError_t prepare_expand_pass() {
 
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s) {
   const size_t smem = expand_dynamic_smem(p.B);
-  if (dtype == C2T_BF16) expand_pass_kernel<true><<<grid, kPassThreads, smem, s>>>(p);
-  else expand_pass_kernel<false><<<grid, kPassThreads, smem, s>>>(p);
+  if (dtype == C2T_BF16) expand_pass_kernel<true><<<grid, kExpandThreads, smem, s>>>(p);
+  else expand_pass_kernel<false><<<grid, kExpandThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 
