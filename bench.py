@@ -99,6 +99,27 @@ class ClockSampler:
                 "samples": len(inside)}
 
 
+# ---------------------------------------------------------------------------- sharding (host logic)
+
+def rank_sequence_base(rank: int, batch_per_rank: int) -> int:
+    """First global sequence id of a rank: ranks own disjoint blocks of `batch_per_rank` sequences."""
+    return rank * batch_per_rank
+
+
+def max_over_ranks(value: float, dist=None, device="cpu") -> float:
+    """The slowest rank's figure (all-reduce MAX); the identity without a process group."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_levels_per_second(world: int, batch_per_rank: int, depth: int, ms_per_step: float) -> float:
+    """Sequence-levels per second of the whole job: every rank advances its own sequences (weak scaling)."""
+    return world * batch_per_rank * depth / (ms_per_step * 1e-3)
+
+
 def make_weights(hidden):
     return c2t_inputs.classifier_weights(hidden, seed=0)
 
@@ -189,7 +210,7 @@ def run_cuda(args) -> None:
                      threshold=w["beta"], hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2, device=local_rank)
     ctx = c2t.Context(cfg)
     Nw = ctx.Nw
-    seq_base = rank * B                                   # every rank owns its own sequences
+    seq_base = rank_sequence_base(rank, B)                # every rank owns its own sequences
     draft = [c2t_inputs.draft_logits(B, F, V, 0, l, torch.bfloat16, device=dev, seq_base=seq_base)
              for l in range(D)]
     target = c2t_inputs.target_logits(B, Nw, V, 0, torch.bfloat16, device=dev, seq_base=seq_base)
@@ -253,12 +274,9 @@ def run_cuda(args) -> None:
     full_ms = [evs[s][2 * l].elapsed_time(evs[s][2 * l + 1]) for s in range(args.steps) for l in range(1, D)]
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total_max = float(t.item())
+    ms_total_max = max_over_ranks(ms_total, dist, dev)
     ms_per_step = ms_total_max / args.steps
-    value = world * B * D / (ms_per_step * 1e-3)
+    value = whole_job_levels_per_second(world, B, D, ms_per_step)
 
     # ---- end to end through the host-buffer entry point (pinned host logits in, results out)
     e2e_steps = max(1, min(args.steps, 5))
@@ -276,10 +294,7 @@ def run_cuda(args) -> None:
     g1.record()
     barrier()
     e2e_ms = max(g0.elapsed_time(g1), (time.perf_counter() - t0) * 1e3) / e2e_steps
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     assert torch.equal(results["accept_len"], accept_len) and torch.equal(results["n_nodes"], n_nodes)
     eb = 2
     h2d = B * V * eb + (D - 1) * B * F * V * eb + B * Nw * V * eb + 2 * B * 4
@@ -319,7 +334,7 @@ def run_cuda(args) -> None:
                    "parallelism": f"dp{world} (independent sequences per rank, no collective)"},
         "us_per_step": ms_per_step * 1e3, "us_per_level": ms_per_step * 1e3 / D,
         "clocks": clocks,
-        "e2e": {"value": world * B * D / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": whole_job_levels_per_second(world, B, D, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "expand_pass_kernel<bf16>", "achieved": achieved, "peak": peak,
