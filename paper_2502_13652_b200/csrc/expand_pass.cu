@@ -96,134 +96,31 @@ __device__ __forceinline__ void combine(float &c, float &S, float &U, float c2, 
   c = C;
 }
 
-// element i of a vector := -2^127 (adds exactly 0 to the sums)
-template <bool BF16>
-__device__ __forceinline__ void mask_element(uint4 &q, int i) {
-  uint32_t *w = reinterpret_cast<uint32_t *>(&q);
-  if (BF16) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if (i == 2 * k) w[k] = (w[k] & 0xFFFF0000u) | 0x0000FF00u;
-      if (i == 2 * k + 1) w[k] = (w[k] & 0x0000FFFFu) | 0xFF000000u;
-    }
-  } else {
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if (i == k) w[k] = __float_as_uint(kLowestF32);
-  }
-}
-
 // ---------------------------------------------------------------- segment state
+
+constexpr int kDefer = 6;          // vectors a thread can set aside per segment
 
 // Shared by the CTA for the segment being streamed.
 struct SegShared {
-  unsigned long long buf[kBufCap];        // keys of every element that met the filter when it was read
-  unsigned long long held[kEWarps];        // per warp: the key held out of the sums
-  uint32_t vals[C2T_MAX_TOPK];            // K largest values seen (orderable form); vals[K-1] is the filter
+  unsigned long long buf[kBufCap];        // keys of all elements at or above the filter
+  unsigned long long held[kEWarps];       // per warp: the key held out of the sums
+  float red[kEWarps][3];                  // per warp: offset c, S, U
   uint32_t warm[kEWarps * C2T_MAX_TOPK];
-  float red[kEWarps][3];
-  float m0;
-  int cnt;
-  int overflow;
+  float thr0;                             // the filter of this segment, fixed once seeded
+  float m0;                               // reference of the streamed sums (largest lane maximum of the first group)
+  int cnt;                                // keys appended to buf
 };
 
 // Per thread.
 struct SegState {
-  Acc acc;
-  float m, c, mw, thr;      // reference, offset -m log2(e), warp's running maximum, top-K filter
-  unsigned long long held;  // warp-uniform
+  Acc acc;                  // sums over the groups that stayed below the filter
+  float c, thr0;            // their offset -m0 log2(e); the filter
+  int n_deferred;           // vectors set aside (may exceed kDefer: then the warp redoes its share)
 };
 
 struct Group {
   uint4 q[4];
 };
-
-// An element at or above the filter: remember its key, and raise the filter if its value is new.
-__device__ __forceinline__ void push_candidate(SegShared &sh, int K, float x, uint32_t tok, float thr) {
-  const int pos = atomicAdd(&sh.cnt, 1);
-  if (pos < kBufCap) sh.buf[pos] = make_key(x, tok);
-  else sh.overflow = 1;
-  if (x > thr) {
-    const uint32_t floor_u = f32_orderable(__float_as_uint(thr));
-    uint32_t carry = f32_orderable(__float_as_uint(x));
-    for (int s = 0; s < K; ++s) {
-      const uint32_t old = atomicMax(&sh.vals[s], carry);
-      if (old < carry) carry = old;
-      if (carry <= floor_u) break;
-    }
-  }
-}
-
-template <bool BF16>
-__device__ __forceinline__ void lane_event(SegShared &sh, int K, const uint4 &q, uint32_t tok0, float thr) {
-  float x[Vec<BF16>::N];
-  Vec<BF16>::unpack(q, x);
-#pragma unroll 1
-  for (int i = 0; i < Vec<BF16>::N; ++i)
-    if (x[i] >= thr) push_candidate(sh, K, x[i], tok0 + i, thr);
-}
-
-// Rare, lane-divergent, out of line: some vector of this thread's group holds an element at or
-// above the filter.  No effect on the sums.
-template <bool BF16>
-__device__ __noinline__ void group_filter_events(SegShared *sh, int K, Group g, int vt, int v1, float thr) {
-  using VT = Vec<BF16>;
-#pragma unroll 1
-  for (int u = 0; u < 4; ++u) {
-    const int v = vt + u * NT;
-    if (v < v1 && VT::vmax(g.q[u]) >= thr) lane_event<BF16>(*sh, K, g.q[u], (uint32_t)v * VT::N, thr);
-  }
-}
-
-// Rare, warp-uniform, out of line: some lane of the warp read an element above the warp's
-// running maximum.  Does everything for this group (filter events, hold-out, sums) and returns
-// the thread's new state.
-template <bool BF16>
-__device__ __noinline__ SegState group_with_new_maximum(SegShared *sh, int K, Group g, int vt, int v1, SegState st) {
-  using VT = Vec<BF16>;
-  const int lane = threadIdx.x & 31;
-#pragma unroll 1
-  for (int u = 0; u < 4; ++u) {
-    const int v = vt + u * NT;
-    const bool valid = v < v1;
-    uint4 q = g.q[u];
-    const float vm = VT::vmax(q);
-    if (valid && vm >= st.thr) lane_event<BF16>(*sh, K, q, (uint32_t)v * VT::N, st.thr);   // before any masking
-    const bool rec = valid && vm > st.mw;
-    if (__any_sync(kFull, rec)) {
-      // the warp's new maximum is held out (as an exact key); the previous one joins lane 0's sums
-      unsigned long long mine = 0ull;
-      int idx = 0;
-      if (rec) {
-        float x[VT::N];
-        VT::unpack(q, x);
-#pragma unroll
-        for (int i = VT::N - 1; i >= 0; --i)
-          if (x[i] == vm) idx = i;
-        mine = make_key(vm, (uint32_t)v * VT::N + idx);
-      }
-      unsigned long long best = mine;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(kFull, best, o);
-        best = other > best ? other : best;
-      }
-      const float new_mw = key_value(best);
-      if (new_mw - st.m > 60.f) {          // keep every summed element within e^60 of the reference
-        const float new_c = -new_mw * kLog2e;
-        acc_rescale(st.acc, st.c, new_c);
-        st.m = new_mw;
-        st.c = new_c;
-      }
-      if (lane == 0 && st.held != 0ull) acc_scalar(st.acc, st.c, key_value(st.held));
-      if (rec && mine == best) mask_element<BF16>(q, idx);
-      st.held = best;
-      st.mw = new_mw;
-    }
-    acc_vector<BF16>(st.acc, q, st.c);     // vectors past the segment hold -2^127: they add 0
-  }
-  return st;
-}
 
 // ---------------------------------------------------------------- segments of a span
 
@@ -365,10 +262,12 @@ __device__ __noinline__ void select_by_rescan(int K, int V, int v_full, const ch
   }
 }
 
-// Warm-up, stage 1 (every warp, no barrier): the warp's K largest lane maxima of a segment's
-// first group, descending, into shared memory.
+// Warm-up, stage 1 (every warp, no barrier): the warp's K largest lane maxima over the first
+// two groups of a segment (the first is in registers, the second has just landed in the ring),
+// descending, into shared memory.
 template <bool BF16>
-__device__ __forceinline__ void warmup_stage1(SegShared &sh, int K, const Group &g, int vt, int v1) {
+__device__ __forceinline__ void warmup_stage1(SegShared &sh, int K, const Group &g, int vt, int v1, int v_full,
+                                              const uint4 *next_slot) {
   using VT = Vec<BF16>;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float lmax = -INFINITY;
@@ -376,6 +275,15 @@ __device__ __forceinline__ void warmup_stage1(SegShared &sh, int K, const Group 
   for (int u = 0; u < 4; ++u) {
     if (vt + u * NT < v1) {
       const float vm = VT::vmax(g.q[u]);
+      if (vm == vm) lmax = fmaxf(lmax, vm);
+    }
+  }
+  cp_async_wait<1>();                      // the group after this one (all but the newest request)
+  const int lim = v1 < v_full ? v1 : v_full;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (vt + (4 + u) * NT < lim) {         // same segment, whole vector: it is in the ring
+      const float vm = VT::vmax(next_slot[threadIdx.x + u * NT]);
       if (vm == vm) lmax = fmaxf(lmax, vm);
     }
   }
@@ -390,8 +298,8 @@ __device__ __forceinline__ void warmup_stage1(SegShared &sh, int K, const Group 
 }
 
 // Warm-up, stage 2 (warp 0, between two barriers): the K-th largest of the union of the sorted
-// per-warp lists seeds the filter (a valid lower bound of the segment's K-th largest element),
-// their maximum becomes the reference of the sums; the candidate buffer is emptied.
+// per-warp lists is the segment's filter (K distinct elements are at or above it, so the K
+// largest elements of the segment all are); the largest is the reference of the streamed sums.
 __device__ __forceinline__ void warmup_stage2(SegShared &sh, int K) {
   const int lane = threadIdx.x & 31;
   int head = 0;
@@ -403,41 +311,159 @@ __device__ __forceinline__ void warmup_stage2(SegShared &sh, int K) {
     const unsigned bal = __ballot_sync(kFull, h == mx);
     if (lane == __ffs(bal) - 1) ++head;
   }
-  if (lane < K) sh.vals[lane] = mx;
   if (lane == 0) {
-    sh.m0 = __uint_as_float(f32_from_orderable(first));
+    sh.thr0 = __uint_as_float(f32_from_orderable(mx));
+    // no data at all (every lane maximum is -inf or NaN): any finite reference will do
+    sh.m0 = first == f32_orderable(0xFF800000u) ? 0.f : __uint_as_float(f32_from_orderable(first));
     sh.cnt = 0;
-    sh.overflow = 0;
   }
 }
 
-__device__ __forceinline__ void state_init(const SegShared &sh, SegState &st) {
+// What a thread set aside while streaming: up to kDefer vectors (data and vector index), in
+// its own places of shared memory, NT entries apart.
+struct DeferSlots {
+  uint4 *data;
+  int *index;
+};
+
+// One vector that met the filter, element by element: keys at or above the filter are
+// appended, everything but the held key is summed with offset cd.
+template <bool BF16>
+__device__ __forceinline__ void careful_vector(SegShared &sh, const uint4 &q, uint32_t tok0, float thr0,
+                                               unsigned long long held, Acc &d, float cd) {
+  float x[Vec<BF16>::N];
+  Vec<BF16>::unpack(q, x);
+#pragma unroll
+  for (int i = 0; i < Vec<BF16>::N; ++i) {
+    const unsigned long long key = make_key(x[i], tok0 + i);
+    if (x[i] >= thr0) {
+      const int pos = atomicAdd(&sh.cnt, 1);
+      if (pos < kBufCap) sh.buf[pos] = key;
+    }
+    if (key != held) acc_scalar(d, cd, x[i]);     // (a NaN element poisons the sums, as it must)
+  }
+}
+
+// the largest key of a vector (NaN elements ignored)
+template <bool BF16>
+__device__ __forceinline__ unsigned long long vector_best_key(const uint4 &q, uint32_t tok0) {
+  float x[Vec<BF16>::N];
+  Vec<BF16>::unpack(q, x);
+  unsigned long long best = 0ull;
+#pragma unroll
+  for (int i = 0; i < Vec<BF16>::N; ++i) {
+    const unsigned long long key = make_key(x[i], tok0 + i);
+    if (x[i] == x[i] && key > best) best = key;
+  }
+  return best;
+}
+
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long other = __shfl_xor_sync(kFull, k, o);
+    k = other > k ? other : k;
+  }
+  return k;
+}
+
+// the thread's streamed sums and the sums of what it resolved become one
+__device__ __forceinline__ void merge_deferred(SegState &st, bool any, float cd, const Acc &d) {
+  float c = st.c, S = st.acc.S0 + st.acc.S1, U = st.acc.U0 + st.acc.U1;
+  if (any) combine(c, S, U, cd, d.S0 + d.S1, d.U0 + d.U1);
+  st.c = c;
+  st.acc.S0 = S; st.acc.S1 = 0.f; st.acc.U0 = U; st.acc.U1 = 0.f;
+}
+
+// Fallback, per warp, for a thread that ran out of places: the warp goes over its whole share
+// of the segment again, from global memory, treating every vector as set aside.
+template <bool BF16>
+__device__ __noinline__ unsigned long long resolve_by_rescan(SegShared *shp, const char *row, int v0t, int v1,
+                                                             int v_full, int V, SegState *stp) {
+  using VT = Vec<BF16>;
+  SegState &st = *stp;
   acc_clear(st.acc);
-  st.m = sh.m0;                                      // warp-uniform reference of the sums
-  st.c = -st.m * kLog2e;
-  st.mw = __uint_as_float(f32_from_orderable(f32_orderable(__float_as_uint(st.m)) - 1u));   // just below m0
-  st.held = 0ull;
+  unsigned long long best = 0ull;
+  for (int v = v0t; __any_sync(kFull, v < v1); v += NT) {
+    if (v >= v1) continue;
+    uint4 q = VT::load(row, v, v_full, V);
+    VT::clamp(q);
+    const unsigned long long k = vector_best_key<BF16>(q, (uint32_t)v * VT::N);
+    best = k > best ? k : best;
+  }
+  const unsigned long long held = warp_max_key(best);
+  Acc d;
+  acc_clear(d);
+  const float cd = -(best ? key_value(best) : 0.f) * kLog2e;
+  for (int v = v0t; v < v1; v += NT) {
+    uint4 q = VT::load(row, v, v_full, V);
+    VT::clamp(q);
+    careful_vector<BF16>(*shp, q, (uint32_t)v * VT::N, st.thr0, held, d, cd);
+  }
+  merge_deferred(st, best != 0ull, cd, d);
+  return held;
+}
+
+// End of a segment, per warp: resolve the vectors that were set aside.  Their elements at or
+// above the filter append their keys; the largest of them all is the warp's held key and stays
+// out of the sums; the rest is summed relative to the thread's own largest deferred value and
+// merged into the thread's streamed sums.  Uses only the warp's own data and the segment's
+// filter, so the result does not depend on timing.
+template <bool BF16>
+__device__ __noinline__ unsigned long long resolve_deferred(SegShared *shp, DeferSlots slots, SegState *stp) {
+  using VT = Vec<BF16>;
+  SegState &st = *stp;
+  const int n = st.n_deferred;
+  unsigned long long best = 0ull;
+#pragma unroll 1
+  for (int i = 0; i < n; ++i) {
+    const unsigned long long k = vector_best_key<BF16>(slots.data[i * NT], (uint32_t)slots.index[i * NT] * VT::N);
+    best = k > best ? k : best;
+  }
+  const unsigned long long held = warp_max_key(best);
+  Acc d;
+  acc_clear(d);
+  const float cd = -(best ? key_value(best) : 0.f) * kLog2e;
+#pragma unroll 1
+  for (int i = 0; i < n; ++i)
+    careful_vector<BF16>(*shp, slots.data[i * NT], (uint32_t)slots.index[i * NT] * VT::N, st.thr0, held, d, cd);
+  merge_deferred(st, best != 0ull, cd, d);
+  return held;
 }
 
 // End of a segment, every warp, before the barrier: the warp's sums (fixed order) and held key.
-__device__ __forceinline__ void publish_warp_sums(SegShared &sh, const SegState &st) {
+__device__ __forceinline__ void publish_warp_sums(SegShared &sh, const SegState &st, unsigned long long held) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float S = st.acc.S0 + st.acc.S1, U = st.acc.U0 + st.acc.U1;
+  float c = st.c, S = st.acc.S0 + st.acc.S1, U = st.acc.U0 + st.acc.U1;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {                   // the offset is warp-uniform: plain sums
-    S += __shfl_down_sync(kFull, S, o);
-    U += __shfl_down_sync(kFull, U, o);
+  for (int o = 16; o > 0; o >>= 1) {                   // offsets may differ between lanes
+    const float c_o = __shfl_down_sync(kFull, c, o);
+    const float S_o = __shfl_down_sync(kFull, S, o);
+    const float U_o = __shfl_down_sync(kFull, U, o);
+    combine(c, S, U, c_o, S_o, U_o);
   }
   if (lane == 0) {
-    sh.red[warp][0] = st.c; sh.red[warp][1] = S; sh.red[warp][2] = U;
-    sh.held[warp] = st.held;
+    sh.red[warp][0] = c; sh.red[warp][1] = S; sh.red[warp][2] = U;
+    sh.held[warp] = held;
   }
 }
 
-// End of a segment, warp 0, after the barrier: merge the warps' sums and emit the partial record.
+// End of a segment, after the barrier: every thread ranks at most two of the collected keys
+// (the K largest go out sorted); warp 0 merges the warps' sums and writes the record.
 __device__ __forceinline__ void emit_partial(SegShared &sh, const PassParams &p, size_t slot, bool overflow) {
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int K = p.K;
+  const int n = sh.cnt < kBufCap ? sh.cnt : kBufCap;
+  if (!overflow) {
+    for (int i = threadIdx.x; i < n; i += NT) {
+      const unsigned long long key = sh.buf[i];
+      int rank = 0;
+      for (int r = 0; r < n; ++r) rank += sh.buf[r] > key;
+      if (rank < K) p.part_keys[slot * K + rank] = key;
+    }
+    for (int r = n + threadIdx.x; r < K; r += NT) p.part_keys[slot * K + r] = 0ull;
+  }
+  if (warp != 0) return;
   float cc = lane < kEWarps ? sh.red[lane][0] : sh.red[0][0];
   float S = lane < kEWarps ? sh.red[lane][1] : 0.f;
   float U = lane < kEWarps ? sh.red[lane][2] : 0.f;
@@ -449,36 +475,20 @@ __device__ __forceinline__ void emit_partial(SegShared &sh, const PassParams &p,
     combine(cc, S, U, c_o, S_o, U_o);
   }
   if (lane < kEWarps) p.part_held[slot * kEWarps + lane] = sh.held[lane];
-  int n_keys = K;
-  if (!overflow) {
-    // the K largest keys of the buffer, sorted, by counting
-    const int n = sh.cnt < kBufCap ? sh.cnt : kBufCap;
-    n_keys = n < K ? n : K;
-    if (n <= 32) {                                      // one key per lane, ranked through shuffles
-      const unsigned long long key = lane < n ? sh.buf[lane] : 0ull;
-      int rank = 0;
-      for (int r = 0; r < n; ++r) rank += __shfl_sync(kFull, key, r) > key;
-      if (lane < n && rank < K) p.part_keys[slot * K + rank] = key;
-    } else {
-      for (int i = lane; i < n; i += 32) {
-        const unsigned long long key = sh.buf[i];
-        int rank = 0;
-        for (int r = 0; r < n; ++r) rank += sh.buf[r] > key;
-        if (rank < K) p.part_keys[slot * K + rank] = key;
-      }
-    }
-    for (int r = n_keys + lane; r < K; r += 32) p.part_keys[slot * K + r] = 0ull;
-  }
-  if (lane == 0) p.part_stats[slot] = make_float4(cc, S, U, __int_as_float(n_keys));
+  if (lane == 0) p.part_stats[slot] = make_float4(cc, S, U, __int_as_float(overflow ? K : (n < K ? n : K)));
 }
 
 template <bool BF16>
 __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_kernel(PassParams p) {
   using VT = Vec<BF16>;
-  extern __shared__ __align__(16) unsigned char s_dyn[];     // ring: 2 slots of 4*NT vectors, then row offsets
+  // dynamic shared memory: the ring (2 slots of 4*NT vectors), the threads' deferred-group places, the row offsets
+  extern __shared__ __align__(16) unsigned char s_dyn[];
   __shared__ SegShared sh;
   uint4 *ring = reinterpret_cast<uint4 *>(s_dyn);
-  int *s_off = reinterpret_cast<int *>(s_dyn + 2 * 4 * NT * sizeof(uint4));
+  DeferSlots slots;
+  slots.data = reinterpret_cast<uint4 *>(s_dyn + 2 * 4 * NT * sizeof(uint4)) + threadIdx.x;
+  slots.index = reinterpret_cast<int *>(s_dyn + (2 * 4 + kDefer) * NT * sizeof(uint4)) + threadIdx.x;
+  int *s_off = reinterpret_cast<int *>(s_dyn + (2 * 4 + kDefer) * NT * sizeof(uint4)) + kDefer * NT;
 
   const int K = p.K;
   const int warp = threadIdx.x >> 5;
@@ -500,24 +510,42 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   take_group<BF16>(g, cur, ring, pt.v_full, p.V);
   prefetch_group(pre, ring, pt.v_full);
   pre.advance(p, s_off, esz);
-  warmup_stage1<BF16>(sh, K, g, cur.tv0 + (int)threadIdx.x, cur.seg.v1);
+  warmup_stage1<BF16>(sh, K, g, cur.tv0 + (int)threadIdx.x, cur.seg.v1, pt.v_full, ring + ((n + 1) & 1u) * 4 * NT);
   __syncthreads();
   if (warp == 0) warmup_stage2(sh, K);
   __syncthreads();
 
   for (;;) {
-    // ---- one segment; its first group is in registers and the filter is seeded
+    // ---- one segment; its first group is in registers and the filter is fixed
     const Segment seg = cur.seg;
     SegState st;
-    state_init(sh, st);
+    acc_clear(st.acc);
+    st.c = -sh.m0 * kLog2e;
+    st.thr0 = sh.thr0;
+    st.n_deferred = 0;
     for (;;) {
+      // a vector with an element at or above the filter is set aside; the others are summed.
+      // Everything summed here is below the filter, hence below the reference: no overflow.
       const int vt = cur.tv0 + (int)threadIdx.x;
-      st.thr = __uint_as_float(f32_from_orderable(*reinterpret_cast<volatile uint32_t *>(&sh.vals[K - 1])));
       const float vm4 = fmaxf(fmaxf(VT::vmax(g.q[0]), VT::vmax(g.q[1])), fmaxf(VT::vmax(g.q[2]), VT::vmax(g.q[3])));
-      if (__any_sync(kFull, vm4 > st.mw && vt < seg.v1)) {
-        st = group_with_new_maximum<BF16>(&sh, K, g, vt, seg.v1, st);
+      if (vm4 >= st.thr0 && vt < seg.v1) {
+        int v = vt;                          // rare: rolled, walking the group by rotation
+#pragma unroll 1
+        for (int u = 0; u < 4; ++u) {
+          if (v < seg.v1 && VT::vmax(g.q[0]) >= st.thr0) {
+            if (st.n_deferred < kDefer) {
+              slots.data[st.n_deferred * NT] = g.q[0];
+              slots.index[st.n_deferred * NT] = v;
+            }
+            ++st.n_deferred;
+          } else {
+            acc_vector<BF16>(st.acc, g.q[0], st.c);
+          }
+          const uint4 t = g.q[0];
+          g.q[0] = g.q[1]; g.q[1] = g.q[2]; g.q[2] = g.q[3]; g.q[3] = t;
+          v += NT;
+        }
       } else {
-        if (vm4 >= st.thr && vt < seg.v1) group_filter_events<BF16>(&sh, K, g, vt, seg.v1, st.thr);
 #pragma unroll
         for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], st.c);
       }
@@ -533,20 +561,27 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       }
       if (last) break;
     }
-    // ---- segment boundary: two barriers; warp 0 closes this segment and seeds the next
-    publish_warp_sums(sh, st);
+    // ---- segment boundary
+    unsigned long long held;
+    if (__any_sync(kFull, st.n_deferred > kDefer))
+      held = resolve_by_rescan<BF16>(&sh, seg.row, seg.v0 + (int)threadIdx.x, seg.v1, pt.v_full, p.V, &st);
+    else
+      held = resolve_deferred<BF16>(&sh, slots, &st);
+    publish_warp_sums(sh, st, held);
     const bool more = cur.valid;
-    if (more) warmup_stage1<BF16>(sh, K, g, cur.tv0 + (int)threadIdx.x, cur.seg.v1);
     __syncthreads();
-    const bool overflow = sh.overflow != 0;
+    const bool overflow = sh.cnt > kBufCap;
     const int split = blockIdx.x - (int)(((long long)seg.a * pt.vec_per_row) / pt.span);
     const size_t slot_id = (size_t)seg.a * p.max_splits + split;
-    if (warp == 0) emit_partial(sh, p, slot_id, overflow);
+    emit_partial(sh, p, slot_id, overflow);
     if (overflow)
       select_by_rescan<BF16>(K, p.V, pt.v_full, seg.row, seg.v0, seg.v1, p.part_keys + slot_id * K, sh.held);
-    if (warp == 0 && more) warmup_stage2(sh, K);
+    if (more)
+      warmup_stage1<BF16>(sh, K, g, cur.tv0 + (int)threadIdx.x, cur.seg.v1, pt.v_full, ring + ((n + 1) & 1u) * 4 * NT);
     __syncthreads();
     if (!more) break;
+    if (warp == 0) warmup_stage2(sh, K);
+    __syncthreads();
   }
   cp_async_wait<0>();
 }
@@ -562,7 +597,8 @@ int max_splits_for(int vocab, int elem_bytes, int grid) {
 }
 
 static size_t expand_dynamic_smem(int B) {
-  return 2 * 4 * (size_t)kExpandThreads * sizeof(uint4) + ((size_t)B + 1) * sizeof(int);
+  return 2 * 4 * (size_t)kExpandThreads * sizeof(uint4) + (size_t)kDefer * kExpandThreads * (sizeof(uint4) + sizeof(int)) +
+         ((size_t)B + 1) * sizeof(int);
 }
 
 cudaError_t prepare_expand_pass() {
