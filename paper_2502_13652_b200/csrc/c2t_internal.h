@@ -37,17 +37,17 @@ constexpr float kNegInfAsFinite = -1.7e38f;   // anything at or below this was -
 constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass
 constexpr int kPassCtasPerSm = 2;
 constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors than this
-// the expand pass runs more, smaller CTAs: no register spills at 80 registers per thread, and
-// while one CTA is at a segment boundary the others on the SM keep streaming
+// the expand pass: every warp is a worker of its own (a span of the rows, its own partial records)
 constexpr int kExpandThreads = 256;
 constexpr int kExpandCtasPerSm = 3;
-constexpr int kHeldPerSlot = kExpandThreads / 32;   // exact keys held out of the fp32 sums, one per warp
+constexpr int kExpandWarps = kExpandThreads / 32;
+constexpr int kHeldPerSlot = 1;       // exact keys held out of the fp32 sums per partial record
 
 // What one launch of the vocabulary pass derived from the device-side row counts.
 struct PassInfo {
   int32_t n_rows;       // active rows
   int32_t vec_per_row;  // 16-byte vectors per row (last one may be ragged)
-  int64_t span;         // vectors per CTA
+  int64_t span;         // vectors per worker (a CTA of the arg-max pass, a warp of the expand pass)
 };
 
 struct PassParams {
@@ -66,7 +66,7 @@ struct PassParams {
   unsigned long long *part_best;
 };
 
-int max_splits_for(int vocab, int elem_bytes, int grid);
+int max_splits_for(int vocab, int elem_bytes, int workers);   // workers: CTAs (arg-max) or warps (expand)
 
 cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
