@@ -24,15 +24,17 @@
 //
 // Top-K.  A vector with an element at or above the filter is not summed but set aside in the
 // warp's queue in shared memory (ballot-ranked places, so the order is fixed).  When the queue
-// is nearly full, and at the end of the segment, the warp drains it: the elements go, one per
-// lane, into the warp's sorted list of the 32 largest keys so far (one key per lane, insertion
-// by shuffle) and into the sums; the largest key of the segment stays out of the sums and is
-// handed on exactly, so the sums keep fp32 relative accuracy with respect to "everything but
-// the maximum" however peaked the row is.  The filter starts as the K-th largest lane maximum
-// of the segment's first two groups (K distinct elements are at or above it) and after every
-// drain is just above the K-th largest value so far: later elements of that value have higher
-// token ids and lose the tie.  Everything depends only on the warp's own data in a fixed
-// order, so the results are reproducible bit for bit.
+// is nearly full, and at the end of the segment, the warp drains it, one element per lane and
+// step: elements below the filter join the sums; the others join a small pool of keys next to
+// the K largest keys found so far, the pool is ranked by counting, the K largest stay and the
+// rest join the sums.  At the end of the segment all of the K largest but the first join the
+// sums too: the segment's largest key stays out and is handed on exactly, so the sums keep fp32
+// relative accuracy with respect to "everything but the maximum" however peaked the row is.
+// The filter starts as the K-th largest lane maximum of the segment's first two groups (K
+// distinct elements are at or above it) and after every drain is just above the K-th largest
+// value so far: later elements of that value have higher token ids and lose the tie.
+// Everything depends only on the warp's own data in a fixed order, so the results are
+// reproducible bit for bit.
 #include "vocab_common.cuh"
 
 namespace c2t {
@@ -44,10 +46,13 @@ constexpr int kQueueCap = 160;                        // vectors a warp can set 
 constexpr int kDrainAt = kQueueCap - kGroupVecs;      // a group always fits behind this many
 
 // What one warp owns in shared memory.
+constexpr int kPool = 64;                             // keys ranked at a time (the K kept ones and up to 32 + 32 - K new)
 struct WarpShared {
   uint4 ring[2][kGroupVecs];
   uint4 qdata[kQueueCap];
   int qindex[kQueueCap];
+  unsigned long long pool[kPool];      // [0, K): the K largest keys so far, sorted (0 = none); behind them the new ones
+  unsigned long long ranked[C2T_MAX_TOPK];
 };
 
 // ---------------------------------------------------------------- sums
@@ -95,7 +100,6 @@ struct SegState {
   float c;                    // warp-uniform offset of the sums, -m log2(e)
   float m;                    // warp-uniform reference value
   float thr;                  // warp-uniform filter
-  unsigned long long mine;    // lane r: the r-th largest key drained so far (0 = none)
   int qn;                     // warp-uniform: vectors in the queue
 };
 
@@ -158,9 +162,9 @@ struct GroupCursor {
 
 // ---------------------------------------------------------------- asynchronous prefetch ring
 
-__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gmem_src) {
-  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+template <int OFF>   // both addresses + OFF bytes
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void *gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0 + %2], [%1 + %2], 16;" ::"r"(smem_dst), "l"(gmem_src), "n"(OFF) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -171,9 +175,19 @@ __device__ __forceinline__ void prefetch_group(const GroupCursor &c, uint4 *slot
   if (c.valid) {
     const int lim = c.seg.v1 < v_full ? c.seg.v1 : v_full;
     const uint4 *src = reinterpret_cast<const uint4 *>(c.seg.row) + c.tv0 + lane;
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (c.tv0 + lane + u * 32 < lim) cp_async_16(slot + lane + u * 32, src + u * 32);
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(slot + lane);
+    if (c.tv0 + kGroupVecs <= lim) {
+      cp_async_16<0>(dst, src);
+      cp_async_16<512>(dst, src);
+      cp_async_16<1024>(dst, src);
+      cp_async_16<1536>(dst, src);
+    } else {
+      const int vt = c.tv0 + lane;
+      if (vt < lim) cp_async_16<0>(dst, src);
+      if (vt + 32 < lim) cp_async_16<512>(dst, src);
+      if (vt + 64 < lim) cp_async_16<1024>(dst, src);
+      if (vt + 96 < lim) cp_async_16<1536>(dst, src);
+    }
   }
   cp_async_commit();
 }
@@ -250,90 +264,85 @@ __device__ __noinline__ float2 segment_warmup(int K, Group g, int vt, int v1, in
 
 // ---------------------------------------------------------------- draining the queue
 
-__device__ __forceinline__ unsigned long long shfl_key(unsigned long long k, int src) {
-  return __shfl_sync(kFull, k, src);
-}
-
-__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const unsigned long long other = __shfl_xor_sync(kFull, k, o);
-    k = other > k ? other : k;
-  }
-  return k;
-}
-
 struct Drained {
   Acc acc;
   float c, m, thr;
-  unsigned long long mine;
 };
 
-// Empties the warp's queue, one element per lane and step: every element is summed except the
-// largest key of the segment so far (the head of the list), and the elements that beat the
-// K-th key of the list are inserted into it.
+// Empties the warp's queue, one element per lane and step.  Elements below the filter are
+// summed.  The others are appended to the pool behind the K largest keys so far; whenever
+// another step might not fit, and at the end, the pool is ranked by counting: the K largest
+// keys stay (sorted, not summed yet), the rest is summed.
 template <bool BF16>
-__device__ __noinline__ Drained drain_queue(const WarpShared *ws, int qn, int K, Acc acc, float c, float m, float thr,
-                                            unsigned long long mine) {
+__device__ __noinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc acc, float c, float m, float thr) {
   constexpr int EPV = Vec<BF16>::N;        // elements per vector
   constexpr int VPS = 32 / EPV;            // vectors per step
   const int lane = threadIdx.x & 31;
+  const unsigned lt_mask = (1u << lane) - 1u;
   const int sub = lane / EPV, e = lane % EPV;
-
-  // the largest key in the queue
-  unsigned long long best = 0ull;
-  for (int base = 0; base < qn; base += VPS) {
-    const int j = base + sub;
-    if (j < qn) {
-      float x;
-      if (BF16) x = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t *>(ws->qdata + j)[e] << 16);
-      else x = reinterpret_cast<const float *>(ws->qdata + j)[e];
-      const unsigned long long key = make_key(x, (uint32_t)ws->qindex[j] * EPV + e);
-      if (x == x && key > best) best = key;
+  int pn = K;
+  for (int base = 0;; base += VPS) {
+    const bool more = base < qn;
+    if (!more || pn > kPool - 32) {
+      // ---- rank the pool: lane l owns keys l and l + 32
+      __syncwarp();
+      const unsigned long long a = lane < pn ? ws->pool[lane] : 0ull;
+      const unsigned long long b = lane + 32 < pn ? ws->pool[lane + 32] : 0ull;
+      if (lane < K) ws->ranked[lane] = 0ull;
+      int ra = 0, rb = 0;
+#pragma unroll 4
+      for (int r = 0; r < pn; ++r) {
+        const unsigned long long kr = ws->pool[r];
+        ra += kr > a;
+        rb += kr > b;
+      }
+      __syncwarp();
+      // the reference follows the largest key before anything of the pool is summed
+      const uint32_t top_hi = (a != 0ull && ra == 0) ? (uint32_t)(a >> 32) : ((b != 0ull && rb == 0) ? (uint32_t)(b >> 32) : 0u);
+      const unsigned owner = __ballot_sync(kFull, top_hi != 0u);
+      if (owner) {
+        const float hm = __uint_as_float(f32_from_orderable(__shfl_sync(kFull, top_hi, __ffs(owner) - 1)));
+        if (hm > m) {
+          const float new_c = -hm * kLog2e;
+          acc_rescale(acc, c, new_c);
+          c = new_c;
+          m = hm;
+        }
+      }
+      if (a != 0ull) {
+        if (ra < K) ws->ranked[ra] = a;
+        else acc_scalar(acc, c, key_value(a));
+      }
+      if (b != 0ull) {
+        if (rb < K) ws->ranked[rb] = b;
+        else acc_scalar(acc, c, key_value(b));
+      }
+      __syncwarp();
+      if (lane < K) ws->pool[lane] = ws->ranked[lane];
+      pn = K;
+      if (!more) break;
     }
-  }
-  const unsigned long long qmax = warp_max_key(best);
-  const unsigned long long old_head = shfl_key(mine, 0);
-  const unsigned long long head = qmax > old_head ? qmax : old_head;
-  if (head != 0ull) {
-    const float hm = key_value(head);
-    if (hm > m) {                          // the reference rises: bring the sums along
-      const float new_c = -hm * kLog2e;
-      acc_rescale(acc, c, new_c);
-      c = new_c;
-      m = hm;
-    }
-  }
-  // the previous head is no longer the maximum: it joins the sums
-  if (old_head != 0ull && head != old_head && lane == 0) acc_scalar(acc, c, key_value(old_head));
-
-  unsigned long long kth = shfl_key(mine, K - 1);
-  for (int base = 0; base < qn; base += VPS) {
     const int j = base + sub;
+    bool cand = false;
     unsigned long long key = 0ull;
     if (j < qn) {
       float x;
       if (BF16) x = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t *>(ws->qdata + j)[e] << 16);
       else x = reinterpret_cast<const float *>(ws->qdata + j)[e];
-      const unsigned long long k = make_key(x, (uint32_t)ws->qindex[j] * EPV + e);
-      if (k != head) acc_scalar(acc, c, x);          // (a NaN element poisons the sums, as it must)
-      if (x == x) key = k;
+      cand = x >= thr;
+      if (cand) key = make_key(x, (uint32_t)ws->qindex[j] * EPV + e);
+      else acc_scalar(acc, c, x);                    // (a NaN element poisons the sums, as it must)
     }
-    unsigned cand = __ballot_sync(kFull, key > kth);
-    while (cand) {
-      const int src = __ffs(cand) - 1;
-      cand &= cand - 1;
-      const unsigned long long k = shfl_key(key, src);
-      unsigned long long up = __shfl_up_sync(kFull, mine, 1);
-      if (lane == 0) up = ~0ull;
-      if (k > mine) mine = k > up ? up : k;          // place k, or take over the neighbour's key
-    }
-    kth = shfl_key(mine, K - 1);
+    const unsigned mask = __ballot_sync(kFull, cand);
+    if (cand) ws->pool[pn + __popc(mask & lt_mask)] = key;
+    pn += __popc(mask);
   }
-  // all of the K largest so far are in the list: from now on only values above its K-th matter
+  __syncwarp();
+  // the list is exact for everything read so far: from now on only values above its K-th matter
+  const unsigned long long kth = ws->pool[K - 1];
   if (kth != 0ull) thr = fmaxf(thr, value_just_above((uint32_t)(kth >> 32)));
   Drained d;
-  d.acc = acc; d.c = c; d.m = m; d.thr = thr; d.mine = mine;
+  d.acc = acc; d.c = c; d.m = m; d.thr = thr;
   return d;
 }
 
@@ -391,26 +400,25 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       st.thr = w.x;
       st.m = w.y;
       st.c = -w.y * kLog2e;
-      st.mine = 0ull;
       st.qn = 0;
+      if (lane < K) ws->pool[lane] = 0ull;
       fresh = false;
     }
     // ---- one group: vectors that meet the filter go to the queue, the others into the sums
+    const bool whole = cur.tv0 + kGroupVecs <= seg.v1;          // no lane is past the segment's end
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const bool hit = VT::vmax(g.q[u]) >= st.thr && vt + u * 32 < seg.v1;
+      const bool hit = VT::vmax(g.q[u]) >= st.thr && (whole || vt + u * 32 < seg.v1);
       const unsigned mask = __ballot_sync(kFull, hit);
       if (mask) {
         if (hit) {
           const int pos = st.qn + __popc(mask & lt_mask);
           ws->qdata[pos] = g.q[u];
           ws->qindex[pos] = vt + u * 32;
-          const uint32_t lo = BF16 ? kLowestBf16x2 : __float_as_uint(kLowestF32);
-          g.q[u] = make_uint4(lo, lo, lo, lo);       // adds exactly 0 below
         }
         st.qn += __popc(mask);
       }
-      acc_vector<BF16>(st.acc, g.q[u], st.c);
+      if (!hit) acc_vector<BF16>(st.acc, g.q[u], st.c);
     }
     const bool last = cur.last_of_segment();
     cur.advance(p, s_off, esz);
@@ -424,13 +432,16 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
     }
     if (last || st.qn > kDrainAt) {
       __syncwarp();                                  // the queue was written by other lanes
-      const Drained d = drain_queue<BF16>(ws, st.qn, K, st.acc, st.c, st.m, st.thr, st.mine);
-      st.acc = d.acc; st.c = d.c; st.m = d.m; st.thr = d.thr; st.mine = d.mine;
+      const Drained d = drain_queue<BF16>(ws, st.qn, K, st.acc, st.c, st.m, st.thr);
+      st.acc = d.acc; st.c = d.c; st.m = d.m; st.thr = d.thr;
       st.qn = 0;
       __syncwarp();
     }
     if (last) {
-      // ---- the segment's record: sums in a fixed order, the sorted keys, the held-out head
+      // ---- the segment's record: the K largest keys but the first join the sums; sums in a
+      // fixed order, the sorted keys, the held-out head
+      const unsigned long long mine = lane < K ? ws->pool[lane] : 0ull;
+      if (lane > 0 && mine != 0ull) acc_scalar(st.acc, st.c, key_value(mine));
       float S = st.acc.S0 + st.acc.S1, U = st.acc.U0 + st.acc.U1;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
@@ -439,12 +450,13 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       }
       const long long split = worker - ((long long)seg.a * vpr) / span;
       const size_t slot_id = (size_t)seg.a * p.max_splits + (size_t)split;
-      const unsigned have = __ballot_sync(kFull, st.mine != 0ull && lane < K);
-      if (lane < K) p.part_keys[slot_id * K + lane] = st.mine;
+      const unsigned have = __ballot_sync(kFull, mine != 0ull);
+      if (lane < K) p.part_keys[slot_id * K + lane] = mine;
       if (lane == 0) {
-        p.part_held[slot_id] = st.mine;
+        p.part_held[slot_id] = mine;
         p.part_stats[slot_id] = make_float4(st.c, S, U, __int_as_float(__popc(have)));
       }
+      __syncwarp();
       if (!cur.valid) break;
       fresh = true;
     }
