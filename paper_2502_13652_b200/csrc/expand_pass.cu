@@ -42,8 +42,8 @@ namespace {
 
 constexpr int kEWarps = kExpandThreads / 32;
 constexpr int kGroupVecs = 128;                       // vectors of one group of a warp
-constexpr int kQueueCap = 160;                        // vectors a warp can set aside before it must drain
-constexpr int kDrainAt = kQueueCap - kGroupVecs;      // a group always fits behind this many
+constexpr int kDrainAt = 12;                          // queued vectors that trigger a drain: early drains keep the filter tight
+constexpr int kQueueCap = kDrainAt + kGroupVecs;      // a whole group always fits behind kDrainAt vectors
 
 // What one warp owns in shared memory.
 constexpr int kPool = 64;                             // keys ranked at a time (the K kept ones and up to 32 + 32 - K new)
@@ -290,11 +290,16 @@ __device__ __noinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc a
       const unsigned long long b = lane + 32 < pn ? ws->pool[lane + 32] : 0ull;
       if (lane < K) ws->ranked[lane] = 0ull;
       int ra = 0, rb = 0;
+      if (pn <= 32) {
 #pragma unroll 4
-      for (int r = 0; r < pn; ++r) {
-        const unsigned long long kr = ws->pool[r];
-        ra += kr > a;
-        rb += kr > b;
+        for (int r = 0; r < pn; ++r) ra += ws->pool[r] > a;
+      } else {
+#pragma unroll 4
+        for (int r = 0; r < pn; ++r) {
+          const unsigned long long kr = ws->pool[r];
+          ra += kr > a;
+          rb += kr > b;
+        }
       }
       __syncwarp();
       // the reference follows the largest key before anything of the pool is summed
@@ -406,19 +411,28 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
     }
     // ---- one group: vectors that meet the filter go to the queue, the others into the sums
     const bool whole = cur.tv0 + kGroupVecs <= seg.v1;          // no lane is past the segment's end
+    float vm[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const bool hit = VT::vmax(g.q[u]) >= st.thr && (whole || vt + u * 32 < seg.v1);
-      const unsigned mask = __ballot_sync(kFull, hit);
-      if (mask) {
-        if (hit) {
-          const int pos = st.qn + __popc(mask & lt_mask);
-          ws->qdata[pos] = g.q[u];
-          ws->qindex[pos] = vt + u * 32;
+    for (int u = 0; u < 4; ++u) vm[u] = VT::vmax(g.q[u]);
+    const bool any_hit = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])) >= st.thr;
+    if (!__any_sync(kFull, any_hit)) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], st.c);
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool hit = vm[u] >= st.thr && (whole || vt + u * 32 < seg.v1);
+        const unsigned mask = __ballot_sync(kFull, hit);
+        if (mask) {
+          if (hit) {
+            const int pos = st.qn + __popc(mask & lt_mask);
+            ws->qdata[pos] = g.q[u];
+            ws->qindex[pos] = vt + u * 32;
+          }
+          st.qn += __popc(mask);
         }
-        st.qn += __popc(mask);
+        if (!hit) acc_vector<BF16>(st.acc, g.q[u], st.c);
       }
-      if (!hit) acc_vector<BF16>(st.acc, g.q[u], st.c);
     }
     const bool last = cur.last_of_segment();
     cur.advance(p, s_off, esz);
