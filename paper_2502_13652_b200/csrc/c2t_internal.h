@@ -38,8 +38,8 @@ constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass
 constexpr int kPassCtasPerSm = 2;
 constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors than this
 // the expand pass: every warp is a worker of its own (a span of the rows, its own partial records)
-constexpr int kExpandThreads = 256;
-constexpr int kExpandCtasPerSm = 3;
+constexpr int kExpandThreads = 768;
+constexpr int kExpandCtasPerSm = 1;
 constexpr int kExpandWarps = kExpandThreads / 32;
 constexpr int kHeldPerSlot = 1;       // exact keys held out of the fp32 sums per partial record
 
