@@ -351,6 +351,46 @@ __device__ __noinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc a
   return d;
 }
 
+// One group: vectors that meet the filter go to the queue, the others into the sums.  WHOLE:
+// no lane is past the segment's end.
+template <bool BF16, bool WHOLE>
+__device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, SegState &st, int vt, int v1,
+                                              unsigned lt_mask) {
+  using VT = Vec<BF16>;
+  float vm[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) vm[u] = VT::vmax(g.q[u]);
+  const bool any_hit = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])) >= st.thr;
+  if (!__any_sync(kFull, any_hit)) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], st.c);
+  } else {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const bool hit = vm[u] >= st.thr && (WHOLE || vt + u * 32 < v1);
+      const unsigned mask = __ballot_sync(kFull, hit);
+      if (mask) {
+        if (hit) {
+          const int pos = st.qn + __popc(mask & lt_mask);
+          ws->qdata[pos] = g.q[u];
+          ws->qindex[pos] = vt + u * 32;
+        }
+        st.qn += __popc(mask);
+      }
+      if (!hit) acc_vector<BF16>(st.acc, g.q[u], st.c);
+    }
+  }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void drain_into(WarpShared *ws, SegState &st, int K) {
+  __syncwarp();                                      // the queue was written by other lanes
+  const Drained d = drain_queue<BF16>(ws, st.qn, K, st.acc, st.c, st.m, st.thr);
+  st.acc = d.acc; st.c = d.c; st.m = d.m; st.thr = d.thr;
+  st.qn = 0;
+  __syncwarp();
+}
+
 // ---------------------------------------------------------------- the kernel
 
 template <bool BF16>
@@ -398,9 +438,8 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   bool fresh = true;                                 // the current group opens a segment
   for (;;) {
     const Segment seg = cur.seg;
-    const int vt = cur.tv0 + lane;
     if (fresh) {
-      const float2 w = segment_warmup<BF16>(K, g, vt, seg.v1, v_full, ws->ring[(n + 1) & 1u]);
+      const float2 w = segment_warmup<BF16>(K, g, cur.tv0 + lane, seg.v1, v_full, ws->ring[(n + 1) & 1u]);
       st.acc.S0 = st.acc.S1 = st.acc.U0 = st.acc.U1 = 0.f;
       st.thr = w.x;
       st.m = w.y;
@@ -409,31 +448,41 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       if (lane < K) ws->pool[lane] = 0ull;
       fresh = false;
     }
-    // ---- one group: vectors that meet the filter go to the queue, the others into the sums
-    const bool whole = cur.tv0 + kGroupVecs <= seg.v1;          // no lane is past the segment's end
-    float vm[4];
+    // ---- the inside of a segment: this group, the next one (in the ring) and the one to be
+    // requested (three ahead) are whole groups of this segment, so nothing needs checking
+    if (pre.valid && pre.seg.a == seg.a) {
+      const int lim = seg.v1 < v_full ? seg.v1 : v_full;
+      const int k = (lim - cur.tv0) / kGroupVecs - 3;
+      if (k > 0) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(seg.row) + pre.tv0 + lane;
+        int vt = cur.tv0 + lane;
+        for (int i = 0; i < k; ++i) {
+          process_group<BF16, true>(ws, g, st, vt, 0, lt_mask);
+          ++n;
+          vt += kGroupVecs;
+          cp_async_wait<1>();
+          uint4 *slot = ws->ring[n & 1u];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) vm[u] = VT::vmax(g.q[u]);
-    const bool any_hit = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])) >= st.thr;
-    if (!__any_sync(kFull, any_hit)) {
+          for (int u = 0; u < 4; ++u) g.q[u] = slot[lane + u * 32];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], st.c);
-    } else {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const bool hit = vm[u] >= st.thr && (whole || vt + u * 32 < seg.v1);
-        const unsigned mask = __ballot_sync(kFull, hit);
-        if (mask) {
-          if (hit) {
-            const int pos = st.qn + __popc(mask & lt_mask);
-            ws->qdata[pos] = g.q[u];
-            ws->qindex[pos] = vt + u * 32;
-          }
-          st.qn += __popc(mask);
+          for (int u = 0; u < 4; ++u) VT::clamp(g.q[u]);
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(slot + lane);
+          cp_async_16<0>(dst, src);
+          cp_async_16<512>(dst, src);
+          cp_async_16<1024>(dst, src);
+          cp_async_16<1536>(dst, src);
+          cp_async_commit();
+          src += kGroupVecs;
+          if (st.qn > kDrainAt) drain_into<BF16>(ws, st, K);
         }
-        if (!hit) acc_vector<BF16>(st.acc, g.q[u], st.c);
+        cur.tv0 += k * kGroupVecs;
+        pre.tv0 += (k - 1) * kGroupVecs;             // the last step may leave the segment
+        pre.advance(p, s_off, esz);
       }
     }
+    // ---- one group near the end of a segment, everything checked
+    const int vt = cur.tv0 + lane;
+    process_group<BF16, false>(ws, g, st, vt, seg.v1, lt_mask);
     const bool last = cur.last_of_segment();
     cur.advance(p, s_off, esz);
     ++n;
@@ -444,13 +493,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       prefetch_group(pre, slot, v_full, lane);
       pre.advance(p, s_off, esz);
     }
-    if (last || st.qn > kDrainAt) {
-      __syncwarp();                                  // the queue was written by other lanes
-      const Drained d = drain_queue<BF16>(ws, st.qn, K, st.acc, st.c, st.m, st.thr);
-      st.acc = d.acc; st.c = d.c; st.m = d.m; st.thr = d.thr;
-      st.qn = 0;
-      __syncwarp();
-    }
+    if (last || st.qn > kDrainAt) drain_into<BF16>(ws, st, K);
     if (last) {
       // ---- the segment's record: the K largest keys but the first join the sums; sums in a
       // fixed order, the sorted keys, the held-out head
