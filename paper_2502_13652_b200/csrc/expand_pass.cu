@@ -78,13 +78,14 @@ __device__ __forceinline__ void acc_scalar(Acc &a, float c, float x) {
   a.U0 = fmaf(e, t, a.U0);
 }
 
+// the sums of one vector; t = x scale + c (scale is log2(e), or 0 to leave the vector out)
 template <bool BF16>
-__device__ __forceinline__ void acc_vector(Acc &a, const uint4 &q, float c) {
+__device__ __forceinline__ void acc_vector(Acc &a, const uint4 &q, float scale, float c) {
   float x[Vec<BF16>::N];
   Vec<BF16>::unpack(q, x);
 #pragma unroll
   for (int i = 0; i < Vec<BF16>::N; i += 2) {
-    const float t0 = fmaf(x[i], kLog2e, c), t1 = fmaf(x[i + 1], kLog2e, c);
+    const float t0 = fmaf(x[i], scale, c), t1 = fmaf(x[i + 1], scale, c);
     const float e0 = ex2f(t0), e1 = ex2f(t1);
     a.S0 += e0;
     a.S1 += e1;
@@ -363,22 +364,29 @@ __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, Se
   const bool any_hit = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])) >= st.thr;
   if (!__any_sync(kFull, any_hit)) {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], st.c);
+    for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], kLog2e, st.c);
   } else {
+    // The sums still run over all four vectors in one straight line; a vector that goes to the
+    // queue is left out by t = 0 x - 200 (2^-200 flushes to zero and 0 * -200 adds nothing to U).
+    bool hit[4];
+    unsigned mask[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const bool hit = vm[u] >= st.thr && (WHOLE || vt + u * 32 < v1);
-      const unsigned mask = __ballot_sync(kFull, hit);
-      if (mask) {
-        if (hit) {
-          const int pos = st.qn + __popc(mask & lt_mask);
-          ws->qdata[pos] = g.q[u];
-          ws->qindex[pos] = vt + u * 32;
-        }
-        st.qn += __popc(mask);
-      }
-      if (!hit) acc_vector<BF16>(st.acc, g.q[u], st.c);
+      hit[u] = vm[u] >= st.thr && (WHOLE || vt + u * 32 < v1);
+      mask[u] = __ballot_sync(kFull, hit[u]);
     }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (hit[u]) {
+        const int pos = st.qn + __popc(mask[u] & lt_mask);
+        ws->qdata[pos] = g.q[u];
+        ws->qindex[pos] = vt + u * 32;
+      }
+      st.qn += __popc(mask[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      acc_vector<BF16>(st.acc, g.q[u], hit[u] ? 0.f : kLog2e, hit[u] ? -200.f : st.c);
   }
 }
 
