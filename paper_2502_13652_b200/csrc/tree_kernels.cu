@@ -10,6 +10,7 @@ constexpr int kTreeThreads = 256;
 constexpr int kTreeWarps = kTreeThreads / 32;
 constexpr int kMaxCand = C2T_MAX_TOPK * C2T_MAX_FRONTIER;   // 1024
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kStageKeys = 256;   // keys of a row's partial lists that a warp stages in shared memory
 
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -84,6 +85,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   __shared__ unsigned char s_keep[kMaxCand], s_sel[kMaxCand];
   __shared__ int s_scan[kTreeWarps + 1];
   __shared__ int s_misc[2];
+  __shared__ unsigned long long s_keys[kTreeWarps][kStageKeys];
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = t.K, F = t.F;
@@ -175,28 +177,52 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
       }
     }
     // the K best keys over all splits become the candidates
-    for (int i = lane; i < n_keys; i += 32) {
-      const unsigned long long key = t.part_keys[slot0 * K + i];
-      if (key == 0ull) continue;
-      const int tok = key_token(key);
-      if (tok >= t.V) continue;                   // padding of a ragged last vector
-      int rank = 0;
-      for (int r = 0; r < n_keys; ++r) {
-        unsigned long long other = t.part_keys[slot0 * K + r];
-        rank += (other > key) && (key_token(other) < t.V);
-      }
-      if (rank < K) { s_x[j * K + rank] = key_value(key); s_tok[j * K + rank] = tok; }
-    }
     S = warp_sum(S);
     T = warp_sum(T);
-    // candidates that do not exist (fewer than K tokens in the vocabulary)
     int n_valid = 0;
-    for (int i = lane; i < n_keys; i += 32) {
-      unsigned long long key = t.part_keys[slot0 * K + i];
-      n_valid += (key != 0ull && key_token(key) < t.V);
-    }
+    if (n_splits <= 32 && n_keys <= kStageKeys) {
+      // every split's list is sorted: stage the lists in shared memory, one per lane, and take
+      // the largest head K times (a key of a token past the vocabulary ends its list: it pads
+      // a ragged last vector and sorts behind every real element)
+      unsigned long long *sk = s_keys[warp];
+      for (int i = lane; i < n_keys; i += 32) sk[i] = t.part_keys[slot0 * K + i];
+      __syncwarp();
+      int pos = 0;
+      for (; n_valid < K; ++n_valid) {
+        unsigned long long h = (lane < n_splits && pos < K) ? sk[lane * K + pos] : 0ull;
+        if (h != 0ull && key_token(h) >= t.V) h = 0ull;
+        unsigned long long mx = h;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) n_valid += __shfl_xor_sync(kFull, n_valid, o);
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long other = __shfl_xor_sync(kFull, mx, o);
+          mx = other > mx ? other : mx;
+        }
+        if (mx == 0ull) break;
+        if (lane == 0) { s_x[j * K + n_valid] = key_value(mx); s_tok[j * K + n_valid] = key_token(mx); }
+        if (h == mx) ++pos;
+      }
+      __syncwarp();
+    } else {
+      for (int i = lane; i < n_keys; i += 32) {
+        const unsigned long long key = t.part_keys[slot0 * K + i];
+        if (key == 0ull) continue;
+        const int tok = key_token(key);
+        if (tok >= t.V) continue;                   // padding of a ragged last vector
+        int rank = 0;
+        for (int r = 0; r < n_keys; ++r) {
+          unsigned long long other = t.part_keys[slot0 * K + r];
+          rank += (other > key) && (key_token(other) < t.V);
+        }
+        if (rank < K) { s_x[j * K + rank] = key_value(key); s_tok[j * K + rank] = tok; }
+      }
+      for (int i = lane; i < n_keys; i += 32) {
+        unsigned long long key = t.part_keys[slot0 * K + i];
+        n_valid += (key != 0ull && key_token(key) < t.V);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) n_valid += __shfl_xor_sync(kFull, n_valid, o);
+    }
+    // candidates that do not exist (fewer than K tokens in the vocabulary)
     for (int r = (n_valid < K ? n_valid : K) + lane; r < K; r += 32) { s_x[j * K + r] = -INFINITY; s_tok[j * K + r] = -1; }
 
     if (lane == 0) {
