@@ -6,11 +6,11 @@
 namespace c2t {
 namespace {
 
-constexpr int kTreeThreads = 256;
+constexpr int kTreeThreads = 512;
 constexpr int kTreeWarps = kTreeThreads / 32;
 constexpr int kMaxCand = C2T_MAX_TOPK * C2T_MAX_FRONTIER;   // 1024
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kStageKeys = 256;   // keys of a row's partial lists that a warp stages in shared memory
+constexpr int kStageKeys = 192;   // keys of a row's partial lists that a warp stages in shared memory
 
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -136,12 +136,27 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     const size_t slot0 = (size_t)a * t.max_splits;
     const int n_keys = n_splits * K;
 
+    // rows with few partials (the usual case): every load is issued before the first use
+    const bool staged = n_splits <= 32 && n_keys <= kStageKeys && kHeldPerSlot == 1;
+    unsigned long long my_held = 0ull;
+    float4 my_stats = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (staged) {
+      if (lane < n_splits) {
+        my_held = t.part_held[slot0 + lane];
+        my_stats = t.part_stats[slot0 + lane];
+      }
+      unsigned long long *sk = s_keys[warp];
+      for (int i = lane; i < n_keys; i += 32) sk[i] = t.part_keys[slot0 * K + i];
+    }
+
     // the row maximum is the largest key held out of any partial's sums
     const int n_held = n_splits * kHeldPerSlot;
-    unsigned long long top = 0ull;
-    for (int i = lane; i < n_held; i += 32) {
-      unsigned long long k0 = t.part_held[slot0 * kHeldPerSlot + i];
-      top = k0 > top ? k0 : top;
+    unsigned long long top = my_held;
+    if (!staged) {
+      for (int i = lane; i < n_held; i += 32) {
+        unsigned long long k0 = t.part_held[slot0 * kHeldPerSlot + i];
+        top = k0 > top ? k0 : top;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -154,7 +169,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     // natural units relative to M:  x - M = t ln2 + g,  g = -c ln2 - M
     double S = 0.0, T = 0.0;
     for (int i = lane; i < n_splits; i += 32) {
-      float4 st = t.part_stats[slot0 + i];
+      const float4 st = staged ? my_stats : t.part_stats[slot0 + i];
       const double Ss = (double)st.y, Us = (double)st.z;
       if (Ss != 0.0 || Us != 0.0) {               // (NaN passes this test and poisons the sums)
         const double kLn2 = 0.69314718055994530942;
@@ -166,7 +181,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     }
     // held-out elements are not in those sums: add them exactly, all but the row maximum itself
     for (int i = lane; i < n_held; i += 32) {
-      const unsigned long long key = t.part_held[slot0 * kHeldPerSlot + i];
+      const unsigned long long key = staged ? my_held : t.part_held[slot0 * kHeldPerSlot + i];
       if (key == 0ull || key == top) continue;
       const float x = key_value(key);
       if (x > kNegInfAsFinite) {
@@ -180,12 +195,11 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     S = warp_sum(S);
     T = warp_sum(T);
     int n_valid = 0;
-    if (n_splits <= 32 && n_keys <= kStageKeys) {
-      // every split's list is sorted: stage the lists in shared memory, one per lane, and take
-      // the largest head K times (a key of a token past the vocabulary ends its list: it pads
-      // a ragged last vector and sorts behind every real element)
-      unsigned long long *sk = s_keys[warp];
-      for (int i = lane; i < n_keys; i += 32) sk[i] = t.part_keys[slot0 * K + i];
+    if (staged) {
+      // every split's list is sorted and now in shared memory, one list per lane: take the
+      // largest head K times (a key of a token past the vocabulary ends its list: it pads a
+      // ragged last vector and sorts behind every real element)
+      const unsigned long long *sk = s_keys[warp];
       __syncwarp();
       int pos = 0;
       for (; n_valid < K; ++n_valid) {
@@ -275,13 +289,14 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   int n_keep;
   block_exclusive_scan(my_keep, s_scan, &n_keep);
   if (n_keep > F) {
-    for (int c = tid; c < nc; c += kTreeThreads) {
+    for (int c = warp; c < nc; c += kTreeWarps) {   // a warp per survivor, its lanes share the comparisons
       if (!s_keep[c]) continue;
       const double Cc = s_C[c];
       int rank = 0;
-      for (int o = 0; o < nc; ++o)
+      for (int o = lane; o < nc; o += 32)
         if (s_keep[o]) rank += (s_C[o] > Cc) || (s_C[o] == Cc && o < c);
-      s_sel[c] = rank < F;
+      rank = __reduce_add_sync(kFull, rank);
+      if (lane == 0) s_sel[c] = rank < F;
     }
   }
   __syncthreads();
