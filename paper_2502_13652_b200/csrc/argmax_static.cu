@@ -89,7 +89,7 @@ extern "C" int c2t_row_argmax_static(const void *logits_dev, int32_t rows, int32
   }
 
   cudaStream_t s = (cudaStream_t)stream;
-  const int max_splits = max_splits_for(vocab, eb, pd.grid);   // <= kStaticMaxSplits by the limits above
+  const int max_splits = max_splits_for(vocab, eb, pd.grid, 0);   // <= kStaticMaxSplits by the limits above
   static_prepare_kernel<<<(rows + 255) / 256, 256, 0, s>>>(pd.scratch, rows, max_splits);
   if (cudaGetLastError() != cudaSuccess) return C2T_ECUDA;
 

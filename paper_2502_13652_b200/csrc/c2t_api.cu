@@ -79,7 +79,7 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   const size_t B = c->batch, F = c->frontier_cap, K = c->topk;
   const size_t cap = tree_capacity_unchecked(c), Nw = c2t_final_width(c);
   const int eb = c->dtype == C2T_BF16 ? 2 : 4;
-  const size_t ms = max_splits_for(c->vocab, eb, kMaxSms * kExpandCtasPerSm * kExpandWarps);   // expand workers outnumber arg-max CTAs
+  const size_t ms = max_splits_for(c->vocab, eb, kMaxSms * kExpandCtasPerSm * kExpandWarps, kSegmentPad);   // expand workers outnumber arg-max CTAs
   TreeState s;
   memset(&s, 0, sizeof s);
   for (int i = 0; i < 2; ++i) {
@@ -186,8 +186,8 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   t.cap = tree_capacity_unchecked(cfg);
   t.hidden = cfg->classifier == C2T_CLS_MLP ? cfg->hidden : 0;
   t.classifier = cfg->classifier; t.tree_add = cfg->tree_add; t.beta = cfg->threshold;
-  t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid_expand * kExpandWarps);
-  t.max_splits_tgt = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid);
+  t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid_expand * kExpandWarps, kSegmentPad);
+  t.max_splits_tgt = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid, 0);
 
   cudaError_t e = cudaSuccess;
   if (cfg->classifier == C2T_CLS_MLP) {

@@ -41,6 +41,11 @@ constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors 
 constexpr int kExpandThreads = 768;
 constexpr int kExpandCtasPerSm = 1;
 constexpr int kExpandWarps = kExpandThreads / 32;
+// Opening a segment (filter warm-up, an extra drain, the record) costs a warp about as much as
+// streaming this many vectors.  The expand pass cuts the rows into spans of equal COST: every row
+// is preceded by this many virtual vectors, the padded rows are laid end to end and cut evenly, and
+// a worker streams the real vectors of its piece.
+constexpr int kSegmentPad = 512;
 constexpr int kHeldPerSlot = 1;       // exact keys held out of the fp32 sums per partial record
 
 // What one launch of the vocabulary pass derived from the device-side row counts.
@@ -48,6 +53,8 @@ struct PassInfo {
   int32_t n_rows;       // active rows
   int32_t vec_per_row;  // 16-byte vectors per row (last one may be ragged)
   int64_t span;         // vectors per worker (a CTA of the arg-max pass, a warp of the expand pass)
+  int32_t pad;          // expand pass: virtual vectors in front of every row (see kSegmentPad), else 0
+  int32_t reserved;
 };
 
 struct PassParams {
@@ -66,7 +73,8 @@ struct PassParams {
   unsigned long long *part_best;
 };
 
-int max_splits_for(int vocab, int elem_bytes, int workers);   // workers: CTAs (arg-max) or warps (expand)
+// partial slots a row can need; workers: CTAs (arg-max, pad 0) or warps (expand, pad kSegmentPad)
+int max_splits_for(int vocab, int elem_bytes, int workers, int pad);
 
 cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);

@@ -3,12 +3,15 @@
 //                                                        (Sec. 4.2.1, Eq. 2, Sec. 4.2.2).
 //
 // Work partition.  The active rows (a device-side count per sequence) are laid end to end as
-// n_rows * vec_per_row 16-byte vectors and cut into equal contiguous spans, one per WARP of a
-// persistent grid (three CTAs of eight warps per SM).  A span may cover the tail of one row and
+// n_rows * vec_per_row 16-byte vectors and cut into contiguous spans of equal cost, one per WARP
+// of a persistent grid (one CTA of 24 warps per SM).  A span may cover the tail of one row and
 // the head of the next; each (row, warp) piece is a "segment" and produces one partial record.
+// Opening a segment costs about as much as streaming kSegmentPad vectors, so the cut is even
+// in vectors + kSegmentPad per row opened.
 // The pruning kernel merges the partials of a row in double precision.  After one barrier at
 // the start (the row list) the warps never wait for each other: while one warp is between
-// segments the other 23 on the SM keep the memory pipe full.
+// segments the other 23 on the SM keep the memory pipe full.  (One CTA per SM rather than
+// three smaller ones: the warps of an older CTA are served first, and its work would end early.)
 //
 // Data movement.  A warp works on groups of 128 consecutive vectors (2 KB), four per lane, 32
 // apart.  Each lane owns 4 x 16 bytes in each of two shared-memory slots and fills them with
@@ -110,6 +113,22 @@ struct Group {
 
 // ---------------------------------------------------------------- segments of a span
 
+// a / b for non-negative operands; the 32-bit division is much shorter when both fit
+__device__ __forceinline__ long long div_floor(long long a, long long b) {
+  if (((unsigned long long)(a | b) >> 32) == 0) return (long long)((unsigned)a / (unsigned)b);
+  return a / b;
+}
+
+// Position x of the padded rows laid end to end -> position in the real rows laid end to end
+// (a position inside a row's pad is the row's start).
+__device__ __forceinline__ long long real_position(long long x, long long vrow, long long vtotal, int vpr) {
+  if (x >= vtotal) x = vtotal;
+  const long long row = div_floor(x, vrow);
+  const long long off = x - row * vrow - kSegmentPad;
+  return row * vpr + (off > 0 ? off : 0);
+}
+
+
 struct Segment {
   const char *row;
   int a, v0, v1;     // vectors [v0, v1) of active row a
@@ -118,7 +137,7 @@ struct Segment {
 struct SegWalk {
   int a, v0, left, vec_per_row;
   __device__ SegWalk(long long start, long long end, int vpr) : vec_per_row(vpr) {
-    a = (int)(start / vpr);
+    a = (int)div_floor(start, vpr);
     v0 = (int)(start - (long long)a * vpr);
     left = (int)(end - start);
   }
@@ -412,18 +431,21 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   const int K = p.K;
   const int n_rows = build_row_offsets(p.counts, p.B, p.rows_per_seq_max, s_off);   // the only barriers
   const int vpr = (p.V + VT::N - 1) / VT::N, v_full = p.V / VT::N;
-  const long long total = (long long)n_rows * vpr;
+  // spans of equal cost: rows behind kSegmentPad virtual vectors each, laid end to end, cut evenly
+  const long long vrow = (long long)vpr + kSegmentPad;
+  const long long vtotal = (long long)n_rows * vrow;
   const long long workers = (long long)gridDim.x * kEWarps;
-  long long span = (total + workers - 1) / workers;
+  long long span = div_floor(vtotal + workers - 1, workers);
   if (span < kMinSpanVectors) span = kMinSpanVectors;
   const long long worker = (long long)blockIdx.x * kEWarps + warp;
   if (worker == 0 && lane == 0) {
     p.info->n_rows = n_rows;
     p.info->vec_per_row = vpr;
     p.info->span = span;
+    p.info->pad = kSegmentPad;
   }
-  const long long start = worker * span;
-  const long long end = start + span < total ? start + span : total;
+  const long long start = real_position(worker * span, vrow, vtotal, vpr);
+  const long long end = real_position((worker + 1) * span, vrow, vtotal, vpr);
   if (start >= end) return;
 
   const size_t esz = BF16 ? 2 : 4;
@@ -513,7 +535,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
         S += __shfl_down_sync(kFull, S, o);
         U += __shfl_down_sync(kFull, U, o);
       }
-      const long long split = worker - ((long long)seg.a * vpr) / span;
+      const long long split = worker - div_floor((long long)seg.a * vrow + kSegmentPad, span);   // workers before the row's first
       const size_t slot_id = (size_t)seg.a * p.max_splits + (size_t)split;
       const unsigned have = __ballot_sync(kFull, mine != 0ull);
       if (lane < K) p.part_keys[slot_id * K + lane] = mine;
@@ -531,10 +553,10 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
 
 }  // namespace
 
-int max_splits_for(int vocab, int elem_bytes, int workers) {
+int max_splits_for(int vocab, int elem_bytes, int workers, int pad) {
   const int vec = 16 / elem_bytes;
   const int vec_per_row = (vocab + vec - 1) / vec;
-  int by_span = (vec_per_row + kMinSpanVectors - 1) / kMinSpanVectors;
+  int by_span = (vec_per_row + pad + kMinSpanVectors - 1) / kMinSpanVectors;
   if (by_span > workers) by_span = workers;
   return by_span + 1;
 }

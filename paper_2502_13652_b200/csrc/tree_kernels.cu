@@ -128,7 +128,8 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   // ---- phase 1: one warp per row merges that row's partial records
   for (int j = warp; j < n; j += kTreeWarps) {
     const int a = row_off + j;
-    const long long first_vec = (long long)a * info.vec_per_row;
+    // the workers that hold a piece of this row: the rows, each behind info.pad virtual vectors, were cut every info.span
+    const long long first_vec = (long long)a * (info.vec_per_row + info.pad) + info.pad;
     const int c_first = (int)(first_vec / info.span);
     const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
     int n_splits = c_last - c_first + 1;

@@ -168,6 +168,7 @@ __device__ __forceinline__ Partition make_partition(const PassParams &p, int n_r
     p.info->n_rows = n_rows;
     p.info->vec_per_row = pt.vec_per_row;
     p.info->span = pt.span;
+    p.info->pad = 0;
   }
   return pt;
 }
