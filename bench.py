@@ -37,6 +37,10 @@ WORKLOAD = dict(B=64, V=128256, D=8, K=10, F=10, N=60, beta=0.5, hidden=16)
 WORKLOAD_NAME = ("B=64 sequences, V=128256, bf16 draft and target logits, depth 8, top-k 10, frontier cap 10, "
                  "budget 60, threshold 0.5, MLP hidden 16")
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one expand_pass_kernel launch at this workload, from the ncu capture summarised in
+# profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  Set to
+# None when the kernel changes until the counters are taken again.
+EXPAND_DRAM_BYTES = {"level0": 16.48e6, "full_level": 171.13e6}
 
 
 def measured_hbm_peak():
@@ -316,6 +320,14 @@ def run_cuda(args) -> None:
         full_bytes = sum(rows_per_level[1:]) * V * eb / (D - 1)
         full_level_gbs = full_bytes / (sum(full_ms) / len(full_ms) * 1e-3) / 1e9
 
+    # DRAM bytes per launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum of this kernel at this workload's
+    # two launch shapes, profiles/expand_pass_kernel_bf16_B64_V128256.txt), scaled by the rows a launch streams
+    # and averaged over the step's launches like `achieved`.  None when the counters do not cover the workload.
+    traffic = None
+    if (B, V, F) == (64, 128256, 10) and EXPAND_DRAM_BYTES is not None:
+        per_row = [EXPAND_DRAM_BYTES["level0"] / 64.0] + [EXPAND_DRAM_BYTES["full_level"] / 640.0] * (D - 1)
+        traffic = sum(r * b for r, b in zip(rows_per_level, per_row)) / D
+
     # ---- the oracle on this host, bounded sample
     n_seq = 8
     dt_cpu, rows_cpu = time_oracle(n_seq, 1, 1)
@@ -339,7 +351,8 @@ def run_cuda(args) -> None:
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "expand_pass_kernel<bf16>", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": None, "bytes_per_launch": bytes_per_launch,
+                     "traffic": traffic, "traffic_unit": "DRAM bytes per launch (ncu, read + write)",
+                     "bytes_per_launch": bytes_per_launch,
                      "avg_launch_us": avg_launch_s * 1e6,
                      "full_level_rows": full_rows, "full_level_gbs": full_level_gbs,
                      "frac_of_8000": achieved / 8000.0},
