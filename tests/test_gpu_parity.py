@@ -251,9 +251,9 @@ def test_call_order_and_alignment_errors():
 
 
 def test_results_are_reproducible():
-    """Every decision (tokens, kept sets, masks, paths) repeats bit for bit; the fp32 tail sums may
-    differ in their last bits between runs, because which thread adds an element evicted from the
-    shared top-K list depends on timing."""
+    """Everything repeats bit for bit, the floating-point results included: every warp of the
+    vocabulary pass works on its own span in a fixed order and the merge adds the partial records
+    in slot order, so no sum depends on timing."""
     B, V, D, K, F, N = 8, 32000, 4, 10, 10, 30
     _, gcfg = make_configs(B, V, D, K, F, N, 0.5, torch.bfloat16)
     Nw = c2t.c2t_final_width(gcfg)
@@ -276,7 +276,7 @@ def test_results_are_reproducible():
         for a, b in zip(snaps[0][0], ints):
             assert torch.equal(a, b)
         for a, b in zip(snaps[0][1], floats):
-            assert torch.allclose(a, b, rtol=1e-6, atol=1e-9)
+            assert torch.equal(a, b)
     ctx.close()
 
 
