@@ -188,6 +188,19 @@ int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride,
                int64_t row_stride, const c2t_accept_out *out, void *stream);
 
 /*
+ * The same greedy acceptance (Sec. 5 Metrics), reading only the target rows the walk visits:
+ * the arg-max of the root's row, then of the accepted child's row, and so on, one row per
+ * sequence and depth, accept_len + 1 rows per sequence instead of all n_nodes.  Arguments,
+ * layout, outputs and error codes are those of c2t_accept; accept_len, path and next_token are
+ * identical to c2t_accept's.  The node_argmax view (c2t_get_view) is filled for the nodes on the
+ * accepted path only, -1 elsewhere.  Issues 2*(D+1)+1 short launches whatever the accept
+ * lengths turn out to be (the host never waits for the device); rounds in which no sequence is
+ * still walking read nothing.  Must follow c2t_prune(C2T_FINAL).
+ */
+int c2t_accept_lazy(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride,
+                    int64_t row_stride, const c2t_accept_out *out, void *stream);
+
+/*
  * The paper has no counterpart to this call; it exists for callers that cannot allocate.
  *
  * Some users of this library may not call cudaMalloc, and may not ask an allocator for a

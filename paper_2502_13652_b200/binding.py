@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.c2t_build_verify.argtypes = [C.c_void_p, P(c2t_verify), C.c_void_p]
         L.c2t_accept.restype = C.c_int
         L.c2t_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, P(c2t_accept_out), C.c_void_p]
+        L.c2t_accept_lazy.restype = C.c_int
+        L.c2t_accept_lazy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, P(c2t_accept_out), C.c_void_p]
         L.c2t_status.restype = C.c_int
         L.c2t_status.argtypes = [C.c_void_p, P(C.c_uint32), C.c_void_p, C.c_void_p]
         L.c2t_get_view.restype = C.c_int
@@ -296,6 +298,14 @@ class Context:
         assert t.shape[0] == self.B and t.shape[2] == self.V and t.stride(2) == 1
         _check(lib().c2t_accept(self._h, t.data_ptr(), t.stride(0), t.stride(1), C.byref(self._accept_c),
                                 _stream(stream)), "c2t_accept")
+
+    def c2t_accept_lazy(self, target_logits: torch.Tensor, stream=None) -> None:
+        """As c2t_accept, reading only the target rows on the accepted path."""
+        t = target_logits
+        assert t.is_cuda and t.dtype == self.cfg.torch_dtype and t.dim() == 3
+        assert t.shape[0] == self.B and t.shape[2] == self.V and t.stride(2) == 1
+        _check(lib().c2t_accept_lazy(self._h, t.data_ptr(), t.stride(0), t.stride(1), C.byref(self._accept_c),
+                                     _stream(stream)), "c2t_accept_lazy")
 
     def c2t_status(self, stream=None):
         """(OR of all status words, per-sequence words as a list).  Synchronises the stream."""

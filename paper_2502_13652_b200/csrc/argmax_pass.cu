@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) argmax_pass_kern
     const int seg = left < (long long)(pt.vec_per_row - v0) ? (int)left : pt.vec_per_row - v0;
     const int v1 = v0 + seg;
     const int b = find_sequence(s_off, p.B, a);
-    const int j = a - s_off[b];
+    const int j = p.row_sel ? p.row_sel[b] : a - s_off[b];
     const char *row = reinterpret_cast<const char *>(p.logits) +
                       ((size_t)b * p.seq_stride + (size_t)j * p.row_stride) * esz;
     const int split = blockIdx.x - (int)(((long long)a * pt.vec_per_row) / pt.span);

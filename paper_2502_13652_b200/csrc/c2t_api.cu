@@ -109,6 +109,9 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   s.node_argmax = w.take<int32_t>(B * Nw);
   s.root_tok = w.take<int32_t>(B);
   s.prefix_len = w.take<int32_t>(B);
+  s.walk_active = w.take<int32_t>(B);
+  s.walk_cur = w.take<int32_t>(B);
+  s.walk_len = w.take<int32_t>(B);
   s.status = w.take<uint32_t>(B);
   s.info_draft = w.take<PassInfo>(1);
   s.info_target = w.take<PassInfo>(1);
@@ -289,6 +292,35 @@ int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, 
     return C2T_ECUDA;
   if (launch_accept_walk(t, out, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
   ctx->launches += 2;
+  return C2T_OK;
+}
+
+int c2t_accept_lazy(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, int64_t row_stride,
+                    const c2t_accept_out *out, void *stream) {
+  if (!ctx || !target_logits_dev) return C2T_EINVAL;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (seq_stride < 0 || row_stride < ctx->cfg.vocab) return C2T_EINVAL;
+  if (!aligned16(target_logits_dev) || (seq_stride * ctx->elem_bytes) % 16 ||
+      (row_stride * ctx->elem_bytes) % 16)
+    return C2T_EALIGN;
+  const TreeState &t = ctx->t;
+  PassParams p;
+  memset(&p, 0, sizeof p);
+  p.logits = target_logits_dev; p.seq_stride = seq_stride; p.row_stride = row_stride;
+  p.V = t.V; p.K = 1; p.B = t.B; p.rows_per_seq_max = 1;
+  p.counts = t.walk_active;          // one row per sequence that is still walking ...
+  p.row_sel = t.walk_cur;            // ... the row of its current node
+  p.max_splits = t.max_splits_tgt;
+  p.info = t.info_target;
+  p.part_best = t.part_best;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (launch_lazy_walk_round(t, 0, out, s) != cudaSuccess) return C2T_ECUDA;
+  ctx->launches += 1;
+  for (int r = 0; r <= t.D; ++r) {   // a path has at most D + 1 nodes
+    if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, s) != cudaSuccess) return C2T_ECUDA;
+    if (launch_lazy_walk_round(t, r + 1, out, s) != cudaSuccess) return C2T_ECUDA;
+    ctx->launches += 2;
+  }
   return C2T_OK;
 }
 

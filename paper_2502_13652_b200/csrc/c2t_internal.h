@@ -63,6 +63,7 @@ struct PassParams {
   int32_t V, K, B;
   int32_t rows_per_seq_max;         // F (draft) or Nw (target)
   const int32_t *counts;            // [B] active rows per sequence, device
+  const int32_t *row_sel;           // arg-max pass only, may be null: [B] the row of sequence b to read (then counts is 0 or 1)
   int32_t max_splits;               // partial slots per row
   PassInfo *info;                   // written by CTA 0
   // expand: per (row, split) partial
@@ -102,6 +103,7 @@ struct TreeState {
   int32_t *final_src, *final_token, *final_parent, *final_level;   // [B, Nw]
   int32_t *node_argmax;        // [B, Nw]
   int32_t *root_tok, *prefix_len;                   // [B]
+  int32_t *walk_active, *walk_cur, *walk_len;       // [B] state of the lazy acceptance walk
   uint32_t *status;            // [B]
   PassInfo *info_draft, *info_target;
   float4 *part_stats;
@@ -117,5 +119,7 @@ cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s);
 cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s);
 cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s);
+// one round of the lazy walk: round 0 starts it, round r > 0 consumes the arg-max of round r-1
+cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s);
 
 }  // namespace c2t

@@ -1,6 +1,8 @@
 // Per-sequence kernels: classification and pruning of a level, the Top-N rerank, the
 // verification inputs and the acceptance walk.  One CTA per sequence; all of this is
 // O(F*K) or O(tree) work per sequence, done in double precision where it is floating point.
+#include <string.h>
+
 #include "c2t_internal.h"
 
 namespace c2t {
@@ -532,7 +534,102 @@ __global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, 
   }
 }
 
+// ---------------------------------------------------------------- lazy walk --
+
+// One round of the acceptance walk that reads only the rows it visits (Sec. 5 Metrics).
+// Round 0 puts every sequence with a tree on its root.  Round r > 0 follows the arg-max pass
+// over the current nodes' rows (one row per walking sequence, in sequence order): the
+// sequence moves to the child that carries the arg-max token, or stops.  A single CTA serves
+// all sequences, 1024 at a time; the scan numbers the walking sequences the way the pass did.
+constexpr int kWalkThreads = 1024;
+
+__global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState t, int round, c2t_accept_out out) {
+  __shared__ int s_warp[kWalkThreads / 32 + 1];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Nw = t.Nw, width = t.D + 1;
+  const PassInfo info = *t.info_target;
+  int rows_before = 0;                               // walking sequences in earlier chunks
+  for (int base = 0; base < t.B; base += kWalkThreads) {
+    const int b = base + tid;
+    const bool in = b < t.B;
+    const size_t fb = (size_t)b * Nw;
+    if (round == 0) {
+      if (in) {
+        const int n = t.final_n[b];
+        for (int i = 0; i < Nw; ++i) t.node_argmax[fb + i] = -1;
+        if (out.path)
+          for (int w = 0; w < width; ++w) out.path[(size_t)b * width + w] = w == 0 ? 0 : -1;
+        t.walk_cur[b] = 0;
+        t.walk_len[b] = 0;
+        t.walk_active[b] = n > 0;
+        if (n <= 0) {
+          if (out.accept_len) out.accept_len[b] = 0;
+          if (out.next_token) out.next_token[b] = -1;
+        }
+      }
+      continue;
+    }
+    const int was = in ? t.walk_active[b] : 0;
+    // the row number of this sequence in the pass: walking sequences before it
+    int inc = was;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += v;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (tid == 0) {
+      int run = 0;
+      for (int w = 0; w < kWalkThreads / 32; ++w) { const int v = s_warp[w]; s_warp[w] = run; run += v; }
+      s_warp[kWalkThreads / 32] = run;
+    }
+    __syncthreads();
+    const int a = rows_before + s_warp[warp] + inc - was;
+    rows_before += s_warp[kWalkThreads / 32];
+    if (!was) continue;
+
+    const long long first_vec = (long long)a * info.vec_per_row;
+    const int c_first = (int)(first_vec / info.span);
+    const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
+    int n_splits = c_last - c_first + 1;
+    if (n_splits > t.max_splits_tgt) n_splits = t.max_splits_tgt;
+    unsigned long long best = 0ull;
+    for (int sp = 0; sp < n_splits; ++sp) {
+      const unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + sp];
+      best = k > best ? k : best;
+    }
+    const int want = best ? key_token(best) : -1;
+    const int n = t.final_n[b];
+    int cur = t.walk_cur[b], len = t.walk_len[b];
+    t.node_argmax[fb + cur] = want;
+    int found = -1;
+    if (len + 1 < width)
+      for (int c = cur + 1; c < n; ++c)
+        if (t.final_parent[fb + c] == cur && t.final_token[fb + c] == want) { found = c; break; }
+    if (found >= 0) {
+      ++len;
+      t.walk_cur[b] = found;
+      t.walk_len[b] = len;
+      if (out.path) out.path[(size_t)b * width + len] = found;
+    } else {
+      t.walk_active[b] = 0;
+      if (out.accept_len) out.accept_len[b] = len;
+      if (out.next_token) out.next_token[b] = want;
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s) {
+  c2t_accept_out o;
+  memset(&o, 0, sizeof o);
+  if (out) o = *out;
+  lazy_walk_round_kernel<<<1, kWalkThreads, 0, s>>>(t, round, o);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
                               cudaStream_t s) {

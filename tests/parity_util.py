@@ -201,6 +201,11 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
     view = {k: v.cpu().numpy() for k, v in ctx.c2t_get_view().items()}
     ver_g = {k: v.cpu().numpy() for k, v in ctx.verify.items()}
     acc_g = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+    # the walk that reads only the rows it visits must give the same answers
+    ctx.c2t_accept_lazy(target_dev)
+    acc_l = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+    amax_l = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+    ctx.c2t_accept(target_dev)                      # leave the all-rows results behind for the caller
     for b in seqs:
         tree, L, ft, ver, acc = orc[b]
         near[b] = near[b] or _near_tie_budget(tree, ocfg.budget)
@@ -231,6 +236,11 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
             ok &= acc_g["accept_len"][b] == acc.accept_len
             ok &= np.array_equal(acc_g["path"][b], acc.path)
             ok &= acc_g["next_token"][b] == acc.next_token
+            ok &= acc_l["accept_len"][b] == acc.accept_len and acc_l["next_token"][b] == acc.next_token
+            ok &= np.array_equal(acc_l["path"][b], acc.path)
+            on_path = np.zeros(ctx.Nw, dtype=bool); on_path[[i for i in acc.path if i >= 0]] = True
+            ok &= np.array_equal(amax_l[b, :m][on_path[:m]], np.asarray(acc.node_argmax[:m])[on_path[:m]])
+            ok &= (amax_l[b][~on_path] == -1).all()
         if not ok and near[b]:
             diverged[b] = True
             continue

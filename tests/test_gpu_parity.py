@@ -280,6 +280,47 @@ def test_results_are_reproducible():
     ctx.close()
 
 
+def test_lazy_accept_follows_planted_paths():
+    """Target rows whose arg-max is planted on a root-to-leaf chain of the final tree: both
+    acceptance calls must walk the whole chain, and the lazy one must not look anywhere else."""
+    B, V, D, K, F, N = 6, 9000, 5, 4, 4, 20
+    dtype = torch.bfloat16
+    _, gcfg = make_configs(B, V, D, K, F, N, 0.0, dtype, classifier="identity")
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype)
+    ctx = c2t.Context(gcfg)
+    ctx.c2t_begin_step(root.cuda(), prefix.cuda())
+    for l in range(D):
+        ctx.c2t_expand_level(l, draft[l].cuda()); ctx.c2t_prune(l)
+    ctx.c2t_prune(c2t.FINAL); ctx.c2t_build_verify()
+    torch.cuda.synchronize()
+    ver = {k: v.cpu().numpy() for k, v in ctx.verify.items()}
+    planted = []
+    for b in range(B):
+        rows = ver["retrieve"][b, :ver["n_leaves"][b]]
+        chain = [int(x) for x in rows[b % len(rows)] if x >= 0]          # a different leaf per sequence
+        for here, nxt in zip(chain, chain[1:]):
+            target[b, here, int(ver["tokens"][b, nxt])] = 100.0
+        if len(chain) < D + 1:                                           # the leaf's own arg-max: a token no child has
+            target[b, chain[-1], V - 1 - b] = 100.0
+        planted.append(chain)
+    tg = target.cuda()
+    ctx.c2t_accept(tg); torch.cuda.synchronize()
+    full = {k: v.cpu().numpy().copy() for k, v in ctx.accepted.items()}
+    amax_full = ctx.c2t_get_view()["node_argmax"].cpu().numpy().copy()
+    ctx.c2t_accept_lazy(tg); torch.cuda.synchronize()
+    lazy = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+    amax_lazy = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+    for b, chain in enumerate(planted):
+        assert full["accept_len"][b] == len(chain) - 1 == lazy["accept_len"][b]
+        assert [x for x in full["path"][b] if x >= 0] == chain == [x for x in lazy["path"][b] if x >= 0]
+        assert full["next_token"][b] == lazy["next_token"][b]
+        for i in range(Nw):
+            assert amax_lazy[b, i] == (amax_full[b, i] if i in chain else -1)
+    assert max(len(c) for c in planted) >= 3
+    ctx.close()
+
+
 def test_decode_step_host_matches_device_path():
     B, V, D, K, F, N = 4, 12000, 4, 6, 5, 16
     _, gcfg = make_configs(B, V, D, K, F, N, 0.5, torch.bfloat16)
