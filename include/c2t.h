@@ -41,8 +41,12 @@ typedef struct c2t_ctx c2t_ctx;
 
 typedef enum { C2T_F32 = 0, C2T_BF16 = 1 } c2t_dtype;
 /* C2T_CLS_MLP: the paper's two-layer FFN.  C2T_CLS_IDENTITY_JOINT: confidence := joint
- * probability, which turns the method into EAGLE-2's expand + rerank (Sec. 2.2). */
-typedef enum { C2T_CLS_MLP = 0, C2T_CLS_IDENTITY_JOINT = 1 } c2t_classifier;
+ * probability, which turns the method into EAGLE-2's expand + rerank (Sec. 2.2) and, with
+ * K = F = 1, into the "DyJoint" early-stop rule of the chain-mode comparison (Sec. 5, Benefits
+ * in Chain Mode).  C2T_CLS_IDENTITY_COND: confidence := the child's own probability under its
+ * parent's distribution; with K = F = 1 the child is the arg-max token, so this is that
+ * comparison's "DyMax" rule (stop when the maximum probability falls below the threshold). */
+typedef enum { C2T_CLS_MLP = 0, C2T_CLS_IDENTITY_JOINT = 1, C2T_CLS_IDENTITY_COND = 2 } c2t_classifier;
 /* What "extend N or topK(N) to T" (Alg. 1) adds to the tree at a level: only the capped
  * next-layer generators, or every node that passed the threshold. */
 typedef enum { C2T_ADD_FRONTIER = 0, C2T_ADD_ALL_SURVIVORS = 1 } c2t_tree_add;

@@ -9,5 +9,5 @@ from .c2t_oracle import (  # noqa: F401
     OracleConfig, LevelRecords, Tree, FinalTree, VerifyInputs, AcceptResult, StepResult,
     build, lib, row_stats, row_softmax, classifier, build_tree, final_prune, build_verify,
     row_argmax, accept, decode_step, tree_capacity, final_width,
-    F32, BF16, CLS_MLP, CLS_IDENTITY_JOINT, ADD_FRONTIER, ADD_ALL_SURVIVORS,
+    F32, BF16, CLS_MLP, CLS_IDENTITY_JOINT, CLS_IDENTITY_COND, ADD_FRONTIER, ADD_ALL_SURVIVORS,
 )

@@ -41,6 +41,7 @@
 
 #define ORC_CLS_MLP 0
 #define ORC_CLS_IDENTITY_JOINT 1
+#define ORC_CLS_IDENTITY_COND 2   /* confidence := the child's own probability ("DyMax" stop rule, chain-mode comparison of Sec. 5) */
 
 #define ORC_ADD_FRONTIER 0
 #define ORC_ADD_ALL_SURVIVORS 1
@@ -268,6 +269,7 @@ int orc_build_tree(const orc_config *cfg, const void *logits, int64_t level_stri
             double C;
             if (ctok[c] < 0 || isnan(clogP[c])) C = NAN;
             else if (cfg->classifier == ORC_CLS_IDENTITY_JOINT) C = P;
+            else if (cfg->classifier == ORC_CLS_IDENTITY_COND) C = exp(clp[c]);
             else C = orc_classifier(P, cH[c], (double)d, cfg->hidden, cfg->w1, cfg->b1, cfg->w2, cfg->b2);
             cC[c] = C;
             ckeep[c] = (C >= cfg->threshold) ? 1 : 0;    /* NaN compares false */

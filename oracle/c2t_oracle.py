@@ -15,7 +15,7 @@ _SRC = os.path.join(_HERE, "c2t_oracle.c")
 _SO = os.path.join(_HERE, "libc2t_oracle.so")
 
 F32, BF16 = 0, 1
-CLS_MLP, CLS_IDENTITY_JOINT = 0, 1
+CLS_MLP, CLS_IDENTITY_JOINT, CLS_IDENTITY_COND = 0, 1, 2
 ADD_FRONTIER, ADD_ALL_SURVIVORS = 0, 1
 
 _lib: Optional[C.CDLL] = None

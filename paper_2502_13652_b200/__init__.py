@@ -7,7 +7,7 @@ from .binding import (  # noqa: F401
     Config, Context, C2TError, lib, LIB_PATH,
     c2t_workspace_bytes, c2t_tree_capacity, c2t_final_width, c2t_mask_words, c2t_row_argmax_static,
     STATIC_MAX_ROWS, STATIC_MAX_VOCAB,
-    F32, BF16, CLS_MLP, CLS_IDENTITY_JOINT, ADD_FRONTIER, ADD_ALL_SURVIVORS, FINAL,
+    F32, BF16, CLS_MLP, CLS_IDENTITY_JOINT, CLS_IDENTITY_COND, ADD_FRONTIER, ADD_ALL_SURVIVORS, FINAL,
     OK, EINVAL, EALIGN, ERANGE, EORDER, ECUDA,
     ST_NAN_LOGIT, ST_POSINF_LOGIT, ST_ALL_NEGINF, ST_TREE_OVERFLOW,
 )

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libc2t.so")
 
 F32, BF16 = 0, 1
-CLS_MLP, CLS_IDENTITY_JOINT = 0, 1
+CLS_MLP, CLS_IDENTITY_JOINT, CLS_IDENTITY_COND = 0, 1, 2
 ADD_FRONTIER, ADD_ALL_SURVIVORS = 0, 1
 FINAL = -1
 OK, EINVAL, EALIGN, ERANGE, EORDER, ECUDA = 0, -1, -2, -3, -4, -5

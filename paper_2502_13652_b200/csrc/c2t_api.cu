@@ -39,7 +39,9 @@ int validate(const c2t_config *c) {
       c->budget < 0 || c->device < 0)
     return C2T_EINVAL;
   if (c->dtype != C2T_F32 && c->dtype != C2T_BF16) return C2T_EINVAL;
-  if (c->classifier != C2T_CLS_MLP && c->classifier != C2T_CLS_IDENTITY_JOINT) return C2T_EINVAL;
+  if (c->classifier != C2T_CLS_MLP && c->classifier != C2T_CLS_IDENTITY_JOINT &&
+      c->classifier != C2T_CLS_IDENTITY_COND)
+    return C2T_EINVAL;
   if (c->tree_add != C2T_ADD_FRONTIER && c->tree_add != C2T_ADD_ALL_SURVIVORS) return C2T_EINVAL;
   if (c->entropy_top_m != 0) return C2T_EINVAL;
   if (!(c->threshold == c->threshold)) return C2T_EINVAL;

@@ -273,6 +273,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     double C;
     if (!ok) C = NAN;
     else if (t.classifier == C2T_CLS_IDENTITY_JOINT) C = P;
+    else if (t.classifier == C2T_CLS_IDENTITY_COND) C = exp(lp);
     else C = classify(t, s_w, P, H, (double)level);
     const bool keep = ok && C >= (double)t.beta;                            // first pruning
     s_C[c] = C;

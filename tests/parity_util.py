@@ -35,13 +35,13 @@ def make_configs(B, V, D, K, F, N, beta, dtype, classifier="mlp", hidden=16, tre
     ocfg = oracle.OracleConfig(
         vocab=V, dtype=oracle.BF16 if dtype == torch.bfloat16 else oracle.F32, max_depth=D, topk=K,
         frontier_cap=F, budget=N, threshold=beta,
-        classifier=oracle.CLS_MLP if classifier == "mlp" else oracle.CLS_IDENTITY_JOINT,
+        classifier={"mlp": oracle.CLS_MLP, "identity": oracle.CLS_IDENTITY_JOINT, "cond": oracle.CLS_IDENTITY_COND}[classifier],
         hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
         tree_add=oracle.ADD_FRONTIER if tree_add == "frontier" else oracle.ADD_ALL_SURVIVORS)
     gcfg = c2t.Config(
         batch=B, vocab=V, dtype=c2t.BF16 if dtype == torch.bfloat16 else c2t.F32, max_depth=D, topk=K,
         frontier_cap=F, budget=N, threshold=beta,
-        classifier=c2t.CLS_MLP if classifier == "mlp" else c2t.CLS_IDENTITY_JOINT,
+        classifier={"mlp": c2t.CLS_MLP, "identity": c2t.CLS_IDENTITY_JOINT, "cond": c2t.CLS_IDENTITY_COND}[classifier],
         hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
         tree_add=c2t.ADD_FRONTIER if tree_add == "frontier" else c2t.ADD_ALL_SURVIVORS)
     return ocfg, gcfg

@@ -116,6 +116,15 @@ def test_chain_mode_k1_f1():
     case(4, 32000, 8, 1, 1, 0, 0.45, torch.bfloat16, wseed=5)
 
 
+@pytest.mark.parametrize("rule,thr", [("cond", 0.3), ("identity", 0.08), ("mlp", 0.5)])
+def test_chain_mode_stop_rules(rule, thr):
+    """K = F = 1 with the three early-stop rules of the chain-mode comparison (Sec. 5): maximum
+    probability, joint probability, the classifier.  Chains end at different depths per sequence."""
+    rep = case(8, 32000, 10, 1, 1, 0, thr, torch.bfloat16, scale=1.5, classifier=rule, wseed=5)
+    assert rep.diverged_sequences == 0 or rep.near_tie_sequences > 0
+    assert len(set(rep.kept_nodes)) >= 2
+
+
 def test_beta_zero_keeps_everything_beta_one_stops_at_root():
     rep = case(2, 4096, 5, 4, 4, 0, 0.0, torch.float32)
     assert rep.kept_nodes == [1 + 4 + 4 * 4] * 2

@@ -218,7 +218,8 @@ def make_cfg(oracle_mod, V, D, K, F, N, beta, classifier="mlp", hidden=16, dtype
     return oracle_mod.OracleConfig(
         vocab=V, dtype=oracle_mod.BF16 if dtype == torch.bfloat16 else oracle_mod.F32,
         max_depth=D, topk=K, frontier_cap=F, budget=N, threshold=beta, entropy_top_m=M,
-        classifier=oracle_mod.CLS_MLP if classifier == "mlp" else oracle_mod.CLS_IDENTITY_JOINT,
+        classifier={"mlp": oracle_mod.CLS_MLP, "identity": oracle_mod.CLS_IDENTITY_JOINT,
+                    "cond": oracle_mod.CLS_IDENTITY_COND}[classifier],
         hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
         tree_add=oracle_mod.ADD_FRONTIER if tree_add == "frontier" else oracle_mod.ADD_ALL_SURVIVORS)
 
@@ -503,6 +504,35 @@ def test_build_tree_chat_is_running_minimum(oracle_mod):
         while a > 0:
             m = min(m, t.C[a]); a = int(t.parent[a])
         assert t.Chat[i] == m
+
+
+# ---------------------------------------------------------------- chain mode --
+
+@pytest.mark.parametrize("rule,thr", [("cond", 0.3), ("identity", 0.08)])
+def test_chain_mode_stop_rules_against_numpy(oracle_mod, rule, thr):
+    """K = F = 1 (Sec. 5, Benefits in Chain Mode): the draft is a chain of arg-max tokens that ends
+    at the first level whose maximum probability ("DyMax", rule cond) or whose joint probability
+    ("DyJoint", rule identity) is below the threshold.  Recomputed here with scipy's softmax."""
+    from scipy.special import softmax
+    V, D = 3000, 8
+    lengths = set()
+    for seq in range(12):
+        cfg = make_cfg(oracle_mod, V, D, 1, 1, 0, thr, classifier=rule)
+        lg = seq_logits(V, D, 1, seq=seq, scale=1.5)
+        t, _ = oracle_mod.build_tree(cfg, lg, 7)
+        want_tok, joint = [], 1.0
+        for l in range(D):
+            p = softmax(lg[l, 0].double().numpy())
+            tok = int(np.argmax(p))                     # (no exact ties in these rows)
+            joint *= p[tok]
+            if (p[tok] if rule == "cond" else joint) < thr:
+                break
+            want_tok.append(tok)
+        assert t.n == 1 + len(want_tok)
+        assert t.tok[1:t.n].tolist() == want_tok
+        assert t.parent[1:t.n].tolist() == list(range(len(want_tok)))
+        lengths.add(len(want_tok))
+    assert len(lengths) >= 3                            # the rule really stops chains at different depths
 
 
 # ---------------------------------------------------------------- verify -----
