@@ -174,6 +174,21 @@ typedef struct {
 /* Tree-attention inputs of the final tree (Sec. 2.2).  Must follow c2t_prune(C2T_FINAL). */
 int c2t_build_verify(c2t_ctx *ctx, const c2t_verify *out, void *stream);
 
+/*
+ * The tree-attention mask (Sec. 2.2) written out as an additive matrix, for attention kernels
+ * that cannot take the bit masks of c2t_build_verify:
+ *   out_dev[b, i, c], i < Nw (c2t_final_width), c < kv_len, of out_dtype (C2T_F32 or C2T_BF16),
+ *   element offset (b*Nw + i)*kv_len + c, caller-owned: 0 where final node i of sequence b
+ *   attends key c, -inf elsewhere.
+ * Keys [0, prefix_len[b]) are the sequence's own prefix, which every row attends; key
+ * prefix_len[b] + j is tree node j, attended iff j is i or an ancestor of i.  Rows i >= n_nodes(b)
+ * attend the prefix only.  Keys at or past kv_len do not exist: the caller chooses
+ * kv_len >= max_b prefix_len[b] + n_nodes(b), or gets a clipped matrix.  prefix_len is the array
+ * given to c2t_begin_step.  Must follow c2t_prune(C2T_FINAL); C2T_EINVAL for kv_len < 1 or an
+ * unknown out_dtype.
+ */
+int c2t_dense_mask(c2t_ctx *ctx, void *out_dev, int32_t out_dtype, int64_t kv_len, void *stream);
+
 typedef struct {
   int32_t *accept_len;   /* [B]      tau of this step: accepted draft tokens, root excluded */
   int32_t *path;         /* [B, D+1] accepted node ids, root first, -1 padded               */

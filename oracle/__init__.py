@@ -7,7 +7,7 @@ baseline do.  It imports nothing from the CUDA package.
 """
 from .c2t_oracle import (  # noqa: F401
     OracleConfig, LevelRecords, Tree, FinalTree, VerifyInputs, AcceptResult, StepResult,
-    build, lib, row_stats, row_softmax, classifier, build_tree, final_prune, build_verify,
+    build, lib, row_stats, row_softmax, classifier, build_tree, final_prune, build_verify, dense_mask,
     row_argmax, accept, decode_step, tree_capacity, final_width,
     F32, BF16, CLS_MLP, CLS_IDENTITY_JOINT, CLS_IDENTITY_COND, ADD_FRONTIER, ADD_ALL_SURVIVORS,
 )

@@ -246,6 +246,24 @@ def build_verify(ft: FinalTree, prefix_len: int, n_rows: int, width: int) -> Ver
     return VerifyInputs(nl, mask, pos, ret)
 
 
+def dense_mask(ft: FinalTree, prefix_len: int, n_rows: int, kv_len: int) -> np.ndarray:
+    """Additive tree-attention mask (Sec. 2.2) written out: [n_rows, kv_len] float64, 0 where final
+    node i attends key c and -inf elsewhere.  Keys [0, prefix_len) are the prefix, which every row
+    attends; key prefix_len + j is tree node j, attended iff j is i or an ancestor of i.  Rows past
+    the tree attend the prefix only.  Keys at or past kv_len do not exist."""
+    out = np.full((n_rows, kv_len), -np.inf)
+    for i in range(n_rows):
+        for c in range(min(int(prefix_len), kv_len)):
+            out[i, c] = 0.0
+        if i < ft.n:
+            j = i
+            while j >= 0:                      # i, its parent, ... up to the root
+                if prefix_len + j < kv_len:
+                    out[i, prefix_len + j] = 0.0
+                j = int(ft.parent[j])
+    return out
+
+
 @dataclass
 class AcceptResult:
     accept_len: int; path: np.ndarray; next_token: int; node_argmax: np.ndarray

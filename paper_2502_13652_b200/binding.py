@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.c2t_build_verify.argtypes = [C.c_void_p, P(c2t_verify), C.c_void_p]
         L.c2t_accept.restype = C.c_int
         L.c2t_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, P(c2t_accept_out), C.c_void_p]
+        L.c2t_dense_mask.restype = C.c_int
+        L.c2t_dense_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_void_p]
         L.c2t_accept_lazy.restype = C.c_int
         L.c2t_accept_lazy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, P(c2t_accept_out), C.c_void_p]
         L.c2t_status.restype = C.c_int
@@ -298,6 +300,14 @@ class Context:
         assert t.shape[0] == self.B and t.shape[2] == self.V and t.stride(2) == 1
         _check(lib().c2t_accept(self._h, t.data_ptr(), t.stride(0), t.stride(1), C.byref(self._accept_c),
                                 _stream(stream)), "c2t_accept")
+
+    def c2t_dense_mask(self, out: torch.Tensor, stream=None) -> None:
+        """out: [B, Nw, kv_len] CUDA tensor, float32 or bfloat16, contiguous: the additive tree-attention mask."""
+        assert out.is_cuda and out.is_contiguous() and out.dim() == 3
+        assert out.shape[0] == self.B and out.shape[1] == self.Nw
+        assert out.dtype in (torch.float32, torch.bfloat16)
+        _check(lib().c2t_dense_mask(self._h, out.data_ptr(), F32 if out.dtype == torch.float32 else BF16,
+                                    out.shape[2], _stream(stream)), "c2t_dense_mask")
 
     def c2t_accept_lazy(self, target_logits: torch.Tensor, stream=None) -> None:
         """As c2t_accept, reading only the target rows on the accepted path."""

@@ -273,6 +273,15 @@ int c2t_build_verify(c2t_ctx *ctx, const c2t_verify *out, void *stream) {
   return C2T_OK;
 }
 
+int c2t_dense_mask(c2t_ctx *ctx, void *out_dev, int32_t out_dtype, int64_t kv_len, void *stream) {
+  if (!ctx || !out_dev || kv_len < 1) return C2T_EINVAL;
+  if (out_dtype != C2T_F32 && out_dtype != C2T_BF16) return C2T_EINVAL;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (launch_dense_mask(ctx->t, out_dev, out_dtype, kv_len, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
+  ctx->launches += 1;
+  return C2T_OK;
+}
+
 int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, int64_t row_stride,
                const c2t_accept_out *out, void *stream) {
   if (!ctx || !target_logits_dev) return C2T_EINVAL;

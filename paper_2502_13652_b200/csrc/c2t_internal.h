@@ -118,6 +118,7 @@ cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const
 cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s);
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s);
 cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s);
+cudaError_t launch_dense_mask(const TreeState &t, void *out, int out_dtype, int64_t kv_len, cudaStream_t s);
 cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s);
 // one round of the lazy walk: round 0 starts it, round r > 0 consumes the arg-max of round r-1
 cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s);

@@ -535,6 +535,34 @@ __global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, 
   }
 }
 
+// ---------------------------------------------------------------- dense mask -
+
+// One CTA per (sequence, final-tree row): the row's ancestor-or-self set as bits in shared
+// memory (a walk up the parent pointers, at most D+1 steps), then the row of kv_len additive
+// mask values, 0 or -inf (Sec. 2.2).
+template <typename T>
+__global__ void __launch_bounds__(256) dense_mask_kernel(TreeState t, T *out, long long kv_len, T zero, T ninf) {
+  __shared__ unsigned long long s_bits[(C2T_MAX_TREE + 63) / 64];   // Nw never exceeds the tree capacity
+  const int b = blockIdx.y, i = blockIdx.x, tid = threadIdx.x;
+  const int Nw = t.Nw, n = t.final_n[b];
+  const int words = (Nw + 63) / 64;
+  for (int w = tid; w < words; w += blockDim.x) s_bits[w] = 0ull;
+  __syncthreads();
+  if (tid == 0 && i < n) {
+    const int32_t *parent = t.final_parent + (size_t)b * Nw;
+    for (int j = i, guard = 0; j >= 0 && guard <= Nw; j = parent[j], ++guard) s_bits[j >> 6] |= 1ull << (j & 63);
+  }
+  __syncthreads();
+  const long long prefix = t.prefix_len[b];
+  T *row = out + ((size_t)b * Nw + i) * kv_len;
+  for (long long c = tid; c < kv_len; c += blockDim.x) {
+    bool on = c < prefix;
+    const long long j = c - prefix;
+    if (j >= 0 && j < Nw) on = (s_bits[j >> 6] >> (j & 63)) & 1ull;
+    row[c] = on ? zero : ninf;
+  }
+}
+
 // ---------------------------------------------------------------- lazy walk --
 
 // One round of the acceptance walk that reads only the rows it visits (Sec. 5 Metrics).
@@ -623,6 +651,18 @@ __global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState
 }
 
 }  // namespace
+
+cudaError_t launch_dense_mask(const TreeState &t, void *out, int out_dtype, int64_t kv_len, cudaStream_t s) {
+  const dim3 grid(t.Nw, t.B);
+  if (out_dtype == C2T_F32) {
+    dense_mask_kernel<float><<<grid, 256, 0, s>>>(t, reinterpret_cast<float *>(out), kv_len, 0.f, -INFINITY);
+  } else {
+    // bf16 as raw 16-bit words: +0 and -inf
+    dense_mask_kernel<unsigned short><<<grid, 256, 0, s>>>(t, reinterpret_cast<unsigned short *>(out), kv_len,
+                                                          (unsigned short)0x0000, (unsigned short)0xFF80);
+  }
+  return cudaGetLastError();
+}
 
 cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s) {
   c2t_accept_out o;

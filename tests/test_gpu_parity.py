@@ -289,6 +289,33 @@ def test_results_are_reproducible():
     ctx.close()
 
 
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_dense_mask_matches_oracle(out_dtype):
+    B, V, D, K, F, N = 5, 6000, 5, 4, 4, 18
+    dtype = torch.bfloat16
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, 0.3, dtype)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype)
+    ctx = c2t.Context(gcfg)
+    ctx.c2t_begin_step(root.cuda(), prefix.cuda())
+    for l in range(D):
+        ctx.c2t_expand_level(l, draft[l].cuda()); ctx.c2t_prune(l)
+    ctx.c2t_prune(c2t.FINAL)
+    for kv_len in (int(prefix.max()) + Nw, int(prefix.max()) + Nw + 13, int(prefix.min()) + 3):   # exact, padded, clipped
+        out = torch.full((B, Nw, kv_len), 7.0, dtype=out_dtype, device="cuda")
+        ctx.c2t_dense_mask(out)
+        got = out.float().cpu().numpy()
+        for b in range(B):
+            lg = torch.stack([draft[l][b] for l in range(D)])
+            tree, _ = oracle.build_tree(ocfg, lg, int(root[b]))
+            ft = oracle.final_prune(tree, N)
+            want = oracle.dense_mask(ft, int(prefix[b]), Nw, kv_len)
+            assert np.array_equal(got[b], want), (b, kv_len)
+    with pytest.raises(c2t.C2TError):
+        ctx.c2t_dense_mask(torch.zeros(B, Nw, 0, device="cuda"))
+    ctx.close()
+
+
 def test_lazy_accept_follows_planted_paths():
     """Target rows whose arg-max is planted on a root-to-leaf chain of the final tree: both
     acceptance calls must walk the whole chain, and the lazy one must not look anywhere else."""

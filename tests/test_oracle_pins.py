@@ -506,6 +506,33 @@ def test_build_tree_chat_is_running_minimum(oracle_mod):
         assert t.Chat[i] == m
 
 
+def test_dense_mask_equals_expanded_bit_masks(oracle_mod):
+    """The dense additive mask is the bit mask of the verify inputs written out behind the prefix:
+    compared entry by entry with the bits (themselves pinned against parent-pointer walks above)."""
+    V, D, K, F, N = 500, 5, 3, 3, 14
+    cfg = make_cfg(oracle_mod, V, D, K, F, N, 0.0, classifier="identity")
+    t, _ = oracle_mod.build_tree(cfg, seq_logits(V, D, F), 3)
+    ft = oracle_mod.final_prune(t, N)
+    Nw, prefix = oracle_mod.final_width(cfg), 7
+    ver = oracle_mod.build_verify(ft, prefix, Nw, D + 1)
+    for kv_len in (prefix + Nw, prefix + Nw + 5, prefix + 4, 3):
+        m = oracle_mod.dense_mask(ft, prefix, Nw, kv_len)
+        assert m.shape == (Nw, kv_len) and set(np.unique(m)) <= {0.0, -np.inf}
+        for i in range(Nw):
+            for c in range(kv_len):
+                if c < prefix:
+                    want = True
+                elif c - prefix < Nw and i < ft.n:
+                    want = bool(int(ver.mask[i, (c - prefix) // 64]) >> ((c - prefix) % 64) & 1)
+                else:
+                    want = False
+                assert (m[i, c] == 0.0) == want
+    # a node attends exactly level+1 tree keys
+    m = oracle_mod.dense_mask(ft, prefix, Nw, prefix + Nw)
+    for i in range(ft.n):
+        assert int((m[i, prefix:] == 0.0).sum()) == int(ft.level[i]) + 1
+
+
 # ---------------------------------------------------------------- chain mode --
 
 @pytest.mark.parametrize("rule,thr", [("cond", 0.3), ("identity", 0.08)])
