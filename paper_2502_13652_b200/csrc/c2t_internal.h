@@ -41,11 +41,12 @@ constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors 
 constexpr int kExpandThreads = 768;
 constexpr int kExpandCtasPerSm = 1;
 constexpr int kExpandWarps = kExpandThreads / 32;
-// Opening a segment (filter warm-up, an extra drain, the record) costs a warp about as much as
-// streaming this many vectors.  The expand pass cuts the rows into spans of equal COST: every row
-// is preceded by this many virtual vectors, the padded rows are laid end to end and cut evenly, and
-// a worker streams the real vectors of its piece.
-constexpr int kSegmentPad = 512;
+// Opening a segment (filter warm-up, extra drains while the filter is still loose, the record)
+// costs a warp about as much as streaming this many vectors (measured: the 640-row level is
+// fastest with 1024 to 2048).  The expand pass cuts the rows into spans of equal COST: every row
+// is preceded by this many virtual vectors, the padded rows are laid end to end and cut evenly,
+// and a worker streams the real vectors of its piece.
+constexpr int kSegmentPad = 1024;
 constexpr int kHeldPerSlot = 1;       // exact keys held out of the fp32 sums per partial record
 
 // What one launch of the vocabulary pass derived from the device-side row counts.
