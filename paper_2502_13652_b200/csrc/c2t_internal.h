@@ -37,8 +37,10 @@ constexpr float kNegInfAsFinite = -1.7e38f;   // anything at or below this was -
 constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass
 constexpr int kPassCtasPerSm = 2;
 constexpr int kMinSpanVectors = 1024; // a CTA never gets fewer 16-byte vectors than this
-// the expand pass: every warp is a worker of its own (a span of the rows, its own partial records)
-constexpr int kExpandThreads = 768;
+// the expand pass: every warp is a worker of its own (a span of the rows, its own partial records).
+// 20 warps per SM: 96 registers per thread (no spills) and fewer segments to open than with 24; measured
+// 3 % faster than 24 warps and 4 % faster than 16.
+constexpr int kExpandThreads = 640;
 constexpr int kExpandCtasPerSm = 1;
 constexpr int kExpandWarps = kExpandThreads / 32;
 // Opening a segment (filter warm-up, extra drains while the filter is still loose, the record)

@@ -4,13 +4,13 @@
 //
 // Work partition.  The active rows (a device-side count per sequence) are laid end to end as
 // n_rows * vec_per_row 16-byte vectors and cut into contiguous spans of equal cost, one per WARP
-// of a persistent grid (one CTA of 24 warps per SM).  A span may cover the tail of one row and
+// of a persistent grid (one CTA of 20 warps per SM).  A span may cover the tail of one row and
 // the head of the next; each (row, warp) piece is a "segment" and produces one partial record.
 // Opening a segment costs about as much as streaming kSegmentPad vectors, so the cut is even
 // in vectors + kSegmentPad per row opened.
 // The pruning kernel merges the partials of a row in double precision.  After one barrier at
 // the start (the row list) the warps never wait for each other: while one warp is between
-// segments the other 23 on the SM keep the memory pipe full.  (One CTA per SM rather than
+// segments the other 19 on the SM keep the memory pipe full.  (One CTA per SM rather than
 // three smaller ones: the warps of an older CTA are served first, and its work would end early.)
 //
 // Data movement.  A warp works on groups of 128 consecutive vectors (2 KB), four per lane, 32
