@@ -437,7 +437,8 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   const long long workers = (long long)gridDim.x * kEWarps;
   long long span = div_floor(vtotal + workers - 1, workers);
   if (span < kMinSpanVectors) span = kMinSpanVectors;
-  const long long worker = (long long)blockIdx.x * kEWarps + warp;
+  // consecutive workers sit on different SMs: a launch with few rows (level 0) still uses every SM
+  const long long worker = (long long)warp * gridDim.x + blockIdx.x;
   if (worker == 0 && lane == 0) {
     p.info->n_rows = n_rows;
     p.info->vec_per_row = vpr;
