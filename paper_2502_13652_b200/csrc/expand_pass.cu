@@ -294,7 +294,7 @@ struct Drained {
 // another step might not fit, and at the end, the pool is ranked by counting: the K largest
 // keys stay (sorted, not summed yet), the rest is summed.
 template <bool BF16>
-__device__ __noinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc acc, float c, float m, float thr) {
+__device__ __forceinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc acc, float c, float m, float thr) {
   constexpr int EPV = Vec<BF16>::N;        // elements per vector
   constexpr int VPS = 32 / EPV;            // vectors per step
   const int lane = threadIdx.x & 31;
