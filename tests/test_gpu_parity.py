@@ -244,6 +244,10 @@ def test_call_order_and_alignment_errors():
     assert code(ctx.c2t_prune, 0) == c2t.EORDER                       # nothing expanded yet
     assert code(ctx.c2t_expand_level, 1, lg) == c2t.EORDER            # wrong level
     assert code(ctx.c2t_build_verify) == c2t.EORDER
+    tg0 = torch.zeros(B, ctx.Nw, V, device="cuda")
+    assert code(ctx.c2t_accept, tg0) == c2t.EORDER                    # no final tree yet
+    assert code(ctx.c2t_accept_lazy, tg0) == c2t.EORDER
+    assert code(ctx.c2t_dense_mask, torch.zeros(B, ctx.Nw, 64, device="cuda")) == c2t.EORDER
     odd = torch.zeros(B * 4 * V + 8, device="cuda")[1:1 + B * 4 * V].view(B, 4, V)
     assert code(ctx.c2t_expand_level, 0, odd) == c2t.EALIGN
     ctx.c2t_expand_level(0, lg)
@@ -253,9 +257,15 @@ def test_call_order_and_alignment_errors():
     ctx.c2t_prune(c2t.FINAL)                                          # fewer than D levels is allowed
     assert code(ctx.c2t_expand_level, 1, lg) == c2t.EORDER            # step is final
     ctx.c2t_build_verify()
-    ctx.c2t_accept(torch.zeros(B, ctx.Nw, V, device="cuda"))
+    ctx.c2t_accept(tg0)
     torch.cuda.synchronize()
-    assert ctx.accepted["accept_len"].tolist() == [0, 0] or True
+    first = {k: v.clone() for k, v in ctx.accepted.items()}
+    ctx.c2t_accept_lazy(tg0)                                          # all-zero rows: arg-max is token 0 everywhere
+    torch.cuda.synchronize()
+    for k, v in ctx.accepted.items():
+        assert torch.equal(v, first[k]), k
+    odd_t = torch.zeros(B * ctx.Nw * V + 8, device="cuda")[1:1 + B * ctx.Nw * V].view(B, ctx.Nw, V)
+    assert code(ctx.c2t_accept_lazy, odd_t) == c2t.EALIGN
     ctx.close()
 
 
