@@ -117,6 +117,7 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   s.status = w.take<uint32_t>(B);
   s.info_draft = w.take<PassInfo>(1);
   s.info_target = w.take<PassInfo>(1);
+  s.row_off_draft = w.take<int32_t>(B + 1);
   s.part_stats = w.take<float4>(B * F * ms);
   s.part_keys = w.take<unsigned long long>(B * F * ms * K);
   s.part_held = w.take<unsigned long long>(B * F * ms * kHeldPerSlot);
@@ -240,6 +241,7 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   p.max_splits = t.max_splits;
   p.info = t.info_draft;
   p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
+  p.row_off = t.row_off_draft;
   if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid_expand, (cudaStream_t)stream) != cudaSuccess)
     return C2T_ECUDA;
   ctx->launches += 1;

@@ -69,6 +69,7 @@ struct PassParams {
   const int32_t *row_sel;           // arg-max pass only, may be null: [B] the row of sequence b to read (then counts is 0 or 1)
   int32_t max_splits;               // partial slots per row
   PassInfo *info;                   // written by CTA 0
+  int32_t *row_off;                 // may be null: [B+1] first active row of every sequence, written by CTA 0
   // expand: per (row, split) partial
   float4 *part_stats;               // {offset c, S, U, n_keys as int bits}: base-2 sums, see expand_pass.cu
   unsigned long long *part_keys;    // [.. * K] the segment's K largest keys, sorted descending, 0-padded
@@ -109,6 +110,7 @@ struct TreeState {
   int32_t *walk_active, *walk_cur, *walk_len;       // [B] state of the lazy acceptance walk
   uint32_t *status;            // [B]
   PassInfo *info_draft, *info_target;
+  int32_t *row_off_draft;          // [B+1] first row of every sequence in the last expand pass
   float4 *part_stats;
   unsigned long long *part_keys;
   unsigned long long *part_held;

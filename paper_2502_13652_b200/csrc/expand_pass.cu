@@ -430,6 +430,8 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
 
   const int K = p.K;
   const int n_rows = build_row_offsets(p.counts, p.B, p.rows_per_seq_max, s_off);   // the only barriers
+  if (blockIdx.x == 0 && p.row_off)                  // the pruning kernel finds a sequence's rows with this
+    for (int i = threadIdx.x; i <= p.B; i += kExpandThreads) p.row_off[i] = s_off[i];
   const int vpr = (p.V + VT::N - 1) / VT::N, v_full = p.V / VT::N;
   // spans of equal cost: rows behind kSegmentPad virtual vectors each, laid end to end, cut evenly
   const long long vrow = (long long)vpr + kSegmentPad;

@@ -88,6 +88,8 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   __shared__ int s_scan[kTreeWarps + 1];
   __shared__ int s_misc[2];
   __shared__ unsigned long long s_keys[kTreeWarps][kStageKeys];
+  unsigned long long *s_ckey = &s_keys[0][0];     // phases 2-3 reuse the staging area: a key per candidate
+  static_assert(kTreeWarps * kStageKeys >= kMaxCand, "candidate keys must fit the staging area");
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = t.K, F = t.F;
@@ -104,17 +106,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     }
     return;
   }
-  // rows of earlier sequences
-  {
-    int part = 0;
-    for (int i = tid; i < b; i += kTreeThreads) {
-      int c = t.frontier_n[cur][i];
-      part += c < 0 ? 0 : (c > F ? F : c);
-    }
-    int total;
-    block_exclusive_scan(part, s_scan, &total);
-    if (tid == 0) s_misc[0] = total;
-  }
+  if (tid == 0) s_misc[1] = 0;                    // survivors of the first pruning
   if (t.classifier == C2T_CLS_MLP) {
     for (int i = tid; i < 3 * t.hidden; i += kTreeThreads) s_w[i] = t.w1[i];
     for (int i = tid; i < t.hidden; i += kTreeThreads) {
@@ -124,7 +116,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     if (tid == 0) s_w[5 * C2T_MAX_HIDDEN] = t.b2[0];
   }
   __syncthreads();
-  const int row_off = s_misc[0];
+  const int row_off = t.row_off_draft[b];         // rows of earlier sequences in the expand pass
   const PassInfo info = *t.info_draft;
 
   // ---- phase 1: one warp per row merges that row's partial records
@@ -208,12 +200,9 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
       for (; n_valid < K; ++n_valid) {
         unsigned long long h = (lane < n_splits && pos < K) ? sk[lane * K + pos] : 0ull;
         if (h != 0ull && key_token(h) >= t.V) h = 0ull;
-        unsigned long long mx = h;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const unsigned long long other = __shfl_xor_sync(kFull, mx, o);
-          mx = other > mx ? other : mx;
-        }
+        const uint32_t hi = (uint32_t)(h >> 32), mx_hi = __reduce_max_sync(kFull, hi);
+        const uint32_t mx_lo = __reduce_max_sync(kFull, hi == mx_hi ? (uint32_t)h : 0u);
+        const unsigned long long mx = ((unsigned long long)mx_hi << 32) | mx_lo;
         if (mx == 0ull) break;
         if (lane == 0) { s_x[j * K + n_valid] = key_value(mx); s_tok[j * K + n_valid] = key_token(mx); }
         if (h == mx) ++pos;
@@ -279,6 +268,10 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     s_C[c] = C;
     s_keep[c] = keep;
     s_sel[c] = keep;
+    // (C desc, index asc) as integer compares: an orderable image of C, 0 for a dropped candidate
+    const unsigned long long cb = (unsigned long long)__double_as_longlong(C);
+    s_ckey[c] = keep ? (cb ^ ((cb >> 63) ? ~0ull : 0x8000000000000000ull)) : 0ull;
+    if (keep) atomicAdd(&s_misc[1], 1);
     t.cand_token[cbase + c] = tok;
     t.cand_lp[cbase + c] = ok ? lp : NAN;
     t.cand_logP[cbase + c] = ok ? logP : NAN;
@@ -288,19 +281,21 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   __syncthreads();
 
   // ---- phase 3: second pruning, the F survivors that come first under (C desc, index asc)
-  int my_keep = 0;
-  for (int c = tid; c < nc; c += kTreeThreads) my_keep += s_keep[c];
-  int n_keep;
-  block_exclusive_scan(my_keep, s_scan, &n_keep);
+  const int n_keep = s_misc[1];
   if (n_keep > F) {
-    for (int c = warp; c < nc; c += kTreeWarps) {   // a warp per survivor, its lanes share the comparisons
-      if (!s_keep[c]) continue;
-      const double Cc = s_C[c];
+    // four threads per survivor share the comparisons against all candidates
+    for (int c0 = 0; c0 < nc; c0 += kTreeThreads / 4) {
+      const int c = c0 + (tid >> 2);
+      const unsigned long long kc = c < nc ? s_ckey[c] : 0ull;
       int rank = 0;
-      for (int o = lane; o < nc; o += 32)
-        if (s_keep[o]) rank += (s_C[o] > Cc) || (s_C[o] == Cc && o < c);
-      rank = __reduce_add_sync(kFull, rank);
-      if (lane == 0) s_sel[c] = rank < F;
+      if (kc != 0ull)
+        for (int o = tid & 3; o < nc; o += 4) {
+          const unsigned long long ko = s_ckey[o];
+          rank += (ko > kc) || (ko == kc && o < c);
+        }
+      rank += __shfl_xor_sync(kFull, rank, 1);
+      rank += __shfl_xor_sync(kFull, rank, 2);
+      if (kc != 0ull && (tid & 3) == 0) s_sel[c] = rank < F;
     }
   }
   __syncthreads();
