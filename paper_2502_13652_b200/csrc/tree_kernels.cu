@@ -95,6 +95,8 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   const int K = t.K, F = t.F;
   const int cur = level & 1, nxt = cur ^ 1;
   int n = t.frontier_n[cur][b];
+  const int row_off = t.row_off_draft[b];         // rows of earlier sequences in the expand pass
+  const PassInfo info = *t.info_draft;            // (loads issued together with the one above)
   n = n < 0 ? 0 : (n > F ? F : n);
   const size_t cbase = (size_t)b * F * K;
 
@@ -116,8 +118,6 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     if (tid == 0) s_w[5 * C2T_MAX_HIDDEN] = t.b2[0];
   }
   __syncthreads();
-  const int row_off = t.row_off_draft[b];         // rows of earlier sequences in the expand pass
-  const PassInfo info = *t.info_draft;
 
   // ---- phase 1: one warp per row merges that row's partial records
   for (int j = warp; j < n; j += kTreeWarps) {
@@ -306,9 +306,11 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   const bool add_all = t.tree_add == C2T_ADD_ALL_SURVIVORS;
   int n_add = 0, n_sel = 0;
   for (int c = c0; c < c1; ++c) { n_add += add_all ? s_keep[c] : s_sel[c]; n_sel += s_sel[c]; }
-  int tot_add, tot_sel;
-  int off_add = block_exclusive_scan(n_add, s_scan, &tot_add);
-  int off_sel = block_exclusive_scan(n_sel, s_scan, &tot_sel);
+  // one scan for both counts (each at most kMaxCand = 1024: 16 bits apiece)
+  int tot_both;
+  const int off_both = block_exclusive_scan(n_add | (n_sel << 16), s_scan, &tot_both);
+  int off_add = off_both & 0xFFFF, off_sel = off_both >> 16;
+  const int tot_add = tot_both & 0xFFFF, tot_sel = tot_both >> 16;
   const int base = t.tree_n[b];
   const bool overflow = base + tot_add > t.cap;
   const size_t tb = (size_t)b * t.cap;
