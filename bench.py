@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one expand_pass_kernel launch at this workload, from the ncu capture summarised in
 # profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  Set to
 # None when the kernel changes until the counters are taken again.
-EXPAND_DRAM_BYTES = {"level0": 16.48e6, "full_level": 168.49e6}
+EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.52e6}
 
 
 def measured_hbm_peak():
