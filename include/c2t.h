@@ -88,7 +88,9 @@ typedef struct {
   int32_t frontier_cap;   /* F                                                            */
   int32_t budget;         /* N, counts the root; 0 = no rerank                            */
   float   threshold;      /* beta; a node is kept iff C >= beta                           */
-  int32_t entropy_top_m;  /* M of Eq. 3; only 0 (exact entropy, Eq. 2) is implemented     */
+  int32_t entropy_top_m;  /* M of Eq. 3: entropy over the M most probable tokens, their
+                             probabilities not renormalised; 0 (or M >= V) = exact, Eq. 2.
+                             M > 0 costs one more pass over the draft logits per level      */
   int32_t classifier;     /* c2t_classifier                                               */
   int32_t hidden;         /* h                                                            */
   const float *w1;        /* HOST [h*3] row-major, features in the order (P, H, d)        */

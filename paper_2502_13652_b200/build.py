@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_HERE, "libc2t.so")
-SOURCES = ["c2t_api.cu", "expand_pass.cu", "argmax_pass.cu", "tree_kernels.cu", "argmax_static.cu"]
+SOURCES = ["c2t_api.cu", "expand_pass.cu", "argmax_pass.cu", "topm_pass.cu", "tree_kernels.cu", "argmax_static.cu"]
 
 
 def _newest_source() -> float:

@@ -43,7 +43,7 @@ int validate(const c2t_config *c) {
       c->classifier != C2T_CLS_IDENTITY_COND)
     return C2T_EINVAL;
   if (c->tree_add != C2T_ADD_FRONTIER && c->tree_add != C2T_ADD_ALL_SURVIVORS) return C2T_EINVAL;
-  if (c->entropy_top_m != 0) return C2T_EINVAL;
+  if (c->entropy_top_m < 0) return C2T_EINVAL;
   if (!(c->threshold == c->threshold)) return C2T_EINVAL;
   if (c->classifier == C2T_CLS_MLP) {
     if (c->hidden < 1 || !c->w1 || !c->b1 || !c->w2 || !c->b2) return C2T_EINVAL;
@@ -118,6 +118,7 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   s.info_draft = w.take<PassInfo>(1);
   s.info_target = w.take<PassInfo>(1);
   s.row_off_draft = w.take<int32_t>(B + 1);
+  s.topm = w.take<double2>(B * F);
   s.part_stats = w.take<float4>(B * F * ms);
   s.part_keys = w.take<unsigned long long>(B * F * ms * K);
   s.part_held = w.take<unsigned long long>(B * F * ms * kHeldPerSlot);
@@ -192,6 +193,7 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   t.cap = tree_capacity_unchecked(cfg);
   t.hidden = cfg->classifier == C2T_CLS_MLP ? cfg->hidden : 0;
   t.classifier = cfg->classifier; t.tree_add = cfg->tree_add; t.beta = cfg->threshold;
+  t.entropy_top_m = cfg->entropy_top_m;
   t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid_expand * kExpandWarps, kSegmentPad);
   t.max_splits_tgt = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid, 0);
 
@@ -245,6 +247,12 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid_expand, (cudaStream_t)stream) != cudaSuccess)
     return C2T_ECUDA;
   ctx->launches += 1;
+  if (t.entropy_top_m > 0 && t.entropy_top_m < t.V) {   // Eq. 3: the sums over the M most probable tokens
+    if (launch_topm_entropy(logits_dev, seq_stride, row_stride, t.V, t.entropy_top_m, t.F, t.B, p.counts, t.topm,
+                            ctx->cfg.dtype, (cudaStream_t)stream) != cudaSuccess)
+      return C2T_ECUDA;
+    ctx->launches += 1;
+  }
   ctx->expanded = 1;
   return C2T_OK;
 }

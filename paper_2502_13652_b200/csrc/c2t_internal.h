@@ -84,6 +84,9 @@ int max_splits_for(int vocab, int elem_bytes, int workers, int pad);
 cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
 cudaError_t launch_argmax_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
+// truncated entropy (Eq. 3): per active row (b, j) the sums over its M largest logits, out[b * F + j] = {S_M, T_M}
+cudaError_t launch_topm_entropy(const void *logits, int64_t seq_stride, int64_t row_stride, int V, int M, int F,
+                                int B, const int32_t *counts, double2 *out, int dtype, cudaStream_t s);
 
 // ---------------------------------------------------------------- tree state -
 
@@ -108,6 +111,8 @@ struct TreeState {
   int32_t *node_argmax;        // [B, Nw]
   int32_t *root_tok, *prefix_len;                   // [B]
   int32_t *walk_active, *walk_cur, *walk_len;       // [B] state of the lazy acceptance walk
+  int32_t entropy_top_m;       // M of Eq. 3 (0: exact entropy)
+  double2 *topm;               // [B, F] {S_M, T_M} of the last expand call when M > 0
   uint32_t *status;            // [B]
   PassInfo *info_draft, *info_target;
   int32_t *row_off_draft;          // [B+1] first row of every sequence in the last expand pass

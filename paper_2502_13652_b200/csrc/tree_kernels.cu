@@ -240,7 +240,12 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
       const double L = log1p(S);                  // ln sum_v e^(x_v - M); the maximum contributes the 1
       s_rowM[j] = M;
       s_rowL[j] = L;
-      s_rowH[j] = L - T / (1.0 + S);              // Eq. 2 with natural log
+      if (t.entropy_top_m > 0 && t.entropy_top_m < t.V) {
+        const double2 sm = t.topm[(size_t)b * F + j];               // Eq. 3: only the M most probable tokens,
+        s_rowH[j] = (L * sm.x - sm.y) / (1.0 + S);                 // probabilities of the full softmax
+      } else {
+        s_rowH[j] = L - T / (1.0 + S);            // Eq. 2 with natural log
+      }
       s_rowfault[j] = (int)fault;
       if (fault) atomicOr(&t.status[b], fault);
     }

@@ -30,17 +30,17 @@ H_ATOL = 1e-12
 
 
 def make_configs(B, V, D, K, F, N, beta, dtype, classifier="mlp", hidden=16, tree_add="frontier",
-                 wseed=0, wstd=0.1, weights=None):
+                 wseed=0, wstd=0.1, weights=None, M=0):
     w1, b1, w2, b2 = weights if weights is not None else c2t_inputs.classifier_weights(hidden, seed=wseed, std=wstd)
     ocfg = oracle.OracleConfig(
         vocab=V, dtype=oracle.BF16 if dtype == torch.bfloat16 else oracle.F32, max_depth=D, topk=K,
-        frontier_cap=F, budget=N, threshold=beta,
+        frontier_cap=F, budget=N, threshold=beta, entropy_top_m=M,
         classifier={"mlp": oracle.CLS_MLP, "identity": oracle.CLS_IDENTITY_JOINT, "cond": oracle.CLS_IDENTITY_COND}[classifier],
         hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
         tree_add=oracle.ADD_FRONTIER if tree_add == "frontier" else oracle.ADD_ALL_SURVIVORS)
     gcfg = c2t.Config(
         batch=B, vocab=V, dtype=c2t.BF16 if dtype == torch.bfloat16 else c2t.F32, max_depth=D, topk=K,
-        frontier_cap=F, budget=N, threshold=beta,
+        frontier_cap=F, budget=N, threshold=beta, entropy_top_m=M,
         classifier={"mlp": c2t.CLS_MLP, "identity": c2t.CLS_IDENTITY_JOINT, "cond": c2t.CLS_IDENTITY_COND}[classifier],
         hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
         tree_add=c2t.ADD_FRONTIER if tree_add == "frontier" else c2t.ADD_ALL_SURVIVORS)

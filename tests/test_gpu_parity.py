@@ -299,6 +299,31 @@ def test_results_are_reproducible():
     ctx.close()
 
 
+@pytest.mark.parametrize("dtype,V,M", [(torch.bfloat16, 32000, 1000), (torch.float32, 32000, 1000),
+                                       (torch.bfloat16, 5000, 100), (torch.float32, 4096, 5),
+                                       (torch.bfloat16, 3000, 3000), (torch.float32, 3000, 7000)])
+def test_truncated_entropy_top_m(dtype, V, M):
+    """Eq. 3: the entropy feature over the M most probable tokens only (the paper's M = 1000), full
+    softmax probabilities; M >= V is the exact entropy again."""
+    rep = case(4, V, 4, 8, 6, 24, 0.5, dtype, M=M)
+    assert rep.diverged_sequences == 0 or rep.near_tie_sequences > 0
+
+
+@pytest.mark.parametrize("kind", ["heavy_ties", "two_valued", "neg_inf", "uniform"])
+def test_truncated_entropy_on_special_rows(kind):
+    """Many equal values around the M-th largest: equal values give equal terms, so only the count matters."""
+    B, V, D, K, F, N = 2, 20000, 2, 5, 4, 10
+    dtype = torch.bfloat16
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, 0.0, dtype, classifier="identity", M=700)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft = [special_rows(kind, B, F, V, dtype) for _ in range(D)]
+    target = special_rows(kind, B, Nw, V, dtype)
+    root = torch.zeros(B, dtype=torch.int32); prefix = torch.full((B,), 9, dtype=torch.int32)
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
+    assert rep.status_bits == 0
+    assert rep.diverged_sequences == 0 or (kind == "uniform" and rep.diverged_sequences <= rep.near_tie_sequences)
+
+
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_dense_mask_matches_oracle(out_dtype):
     B, V, D, K, F, N = 5, 6000, 5, 4, 4, 18

@@ -57,7 +57,7 @@ def test_sizes(L):
 
 @pytest.mark.parametrize("bad,code", [
     (dict(batch=0), c2t.EINVAL), (dict(vocab=0), c2t.EINVAL), (dict(dtype=7), c2t.EINVAL),
-    (dict(classifier=3), c2t.EINVAL), (dict(tree_add=2), c2t.EINVAL), (dict(entropy_top_m=1000), c2t.EINVAL),
+    (dict(classifier=3), c2t.EINVAL), (dict(tree_add=2), c2t.EINVAL), (dict(entropy_top_m=-1), c2t.EINVAL),
     (dict(w1=None), c2t.EINVAL), (dict(threshold=float("nan")), c2t.EINVAL),
     (dict(topk=33), c2t.ERANGE), (dict(frontier_cap=33), c2t.ERANGE), (dict(hidden=65), c2t.ERANGE),
     (dict(budget=1025), c2t.ERANGE), (dict(batch=4097), c2t.ERANGE), (dict(max_depth=33), c2t.ERANGE),
