@@ -176,7 +176,10 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   if (workspace_bytes < carve(cfg, nullptr, nullptr)) return C2T_ERANGE;
   if (cudaSetDevice(cfg->device) != cudaSuccess) { cudaGetLastError(); return C2T_ECUDA; }
   const int grid = pass_grid(cfg->device);
-  if (grid < 0 || prepare_expand_pass() != cudaSuccess) { cudaGetLastError(); return C2T_ECUDA; }
+  if (grid < 0 || prepare_expand_pass() != cudaSuccess || prepare_topm_pass() != cudaSuccess) {
+    cudaGetLastError();
+    return C2T_ECUDA;
+  }
 
   c2t_ctx *ctx = new (std::nothrow) c2t_ctx;
   if (!ctx) return C2T_EINVAL;
@@ -248,7 +251,7 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
     return C2T_ECUDA;
   ctx->launches += 1;
   if (t.entropy_top_m > 0 && t.entropy_top_m < t.V) {   // Eq. 3: the sums over the M most probable tokens
-    if (launch_topm_entropy(logits_dev, seq_stride, row_stride, t.V, t.entropy_top_m, t.F, t.B, p.counts, t.topm,
+    if (launch_topm_entropy(logits_dev, seq_stride, row_stride, t.V, t.entropy_top_m, t.F, t.B, p.counts, t, t.topm,
                             ctx->cfg.dtype, (cudaStream_t)stream) != cudaSuccess)
       return C2T_ECUDA;
     ctx->launches += 1;

@@ -84,10 +84,6 @@ int max_splits_for(int vocab, int elem_bytes, int workers, int pad);
 cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
 cudaError_t launch_argmax_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
-// truncated entropy (Eq. 3): per active row (b, j) the sums over its M largest logits, out[b * F + j] = {S_M, T_M}
-cudaError_t launch_topm_entropy(const void *logits, int64_t seq_stride, int64_t row_stride, int V, int M, int F,
-                                int B, const int32_t *counts, double2 *out, int dtype, cudaStream_t s);
-
 // ---------------------------------------------------------------- tree state -
 
 struct TreeState {
@@ -123,6 +119,12 @@ struct TreeState {
   float *w1, *b1, *w2, *b2;
 };
 
+// truncated entropy (Eq. 3): per active row (b, j) the sums over its M largest logits, out[b * F + j] = {S_M, T_M};
+// runs after the expand pass of the same level, whose partial records give it the row maxima
+cudaError_t prepare_topm_pass();     // once per device: opt in to the kernel's shared-memory size
+cudaError_t launch_topm_entropy(const void *logits, int64_t seq_stride, int64_t row_stride, int V, int M, int F,
+                                int B, const int32_t *counts, const TreeState &t, double2 *out, int dtype,
+                                cudaStream_t s);
 cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
                               cudaStream_t s);
 cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s);
