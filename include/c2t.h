@@ -128,6 +128,8 @@ int c2t_begin_step(c2t_ctx *ctx, const int32_t *root_tok_dev, const int32_t *pre
  * for every active frontier slot (b, j), j < n_level(b), one pass over logits row (b, j)
  * yields the softmax normaliser, the exact entropy of the row and its K most probable
  * tokens (ties to the lower token id).  Results stay in the workspace for c2t_prune.
+ * With cfg.entropy_top_m = M, 0 < M < V, a second kernel reads the active rows once more for
+ * the entropy over the M most probable tokens (Eq. 3) that c2t_prune then uses instead.
  *   logits_dev: [B, F, V] of cfg.dtype; element offset of (b, j, v) =
  *               b*seq_stride + j*row_stride + v.  Base address 16-byte aligned, both strides
  *               multiples of 16 bytes.  Rows of inactive slots are never read.
