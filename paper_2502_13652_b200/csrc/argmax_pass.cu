@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) argmax_pass_kern
   __shared__ unsigned long long s_best[kWarps];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  chain_enter();
   const int n_rows = build_row_offsets(p.counts, p.B, p.rows_per_seq_max, s_off);
   const Partition pt = make_partition<VT::N>(p, n_rows);
   if (pt.start >= pt.end) return;
@@ -91,9 +92,8 @@ __global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) argmax_pass_kern
 }  // namespace
 
 cudaError_t launch_argmax_pass(const PassParams &p, int dtype, int grid, cudaStream_t s) {
-  if (dtype == C2T_BF16) argmax_pass_kernel<true><<<grid, kPassThreads, 0, s>>>(p);
-  else argmax_pass_kernel<false><<<grid, kPassThreads, 0, s>>>(p);
-  return cudaGetLastError();
+  if (dtype == C2T_BF16) return launch_chained(argmax_pass_kernel<true>, dim3(grid), dim3(kPassThreads), 0, s, p);
+  return launch_chained(argmax_pass_kernel<false>, dim3(grid), dim3(kPassThreads), 0, s, p);
 }
 
 }  // namespace c2t

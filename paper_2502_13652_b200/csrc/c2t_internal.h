@@ -32,6 +32,38 @@ __device__ __forceinline__ int32_t key_token(unsigned long long k) {
 // never produces inf - inf or 0 * inf in the running sums.
 constexpr float kNegInfAsFinite = -1.7e38f;   // anything at or below this was -inf (or as good as)
 
+// ---------------------------------------------------------------- launch chain
+// The kernels of a decode step form a chain in which each one consumes what the one before wrote.
+// They are launched with programmatic stream serialisation: the next kernel's CTAs may be placed
+// on SMs (and its launch latency paid) while the previous kernel is still finishing.  Every kernel
+// of the chain therefore starts with chain_enter(): it lets its own successor be scheduled and then
+// waits until the predecessor has completed and its writes are visible.  Nothing touches global
+// memory before that, so the chain behaves exactly like plain stream order.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_enter() {
+  chain_release();
+  chain_wait();
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                           Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // ---------------------------------------------------------------- vocab pass -
 
 constexpr int kPassThreads = 512;     // threads per CTA of the vocabulary pass

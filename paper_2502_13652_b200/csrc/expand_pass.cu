@@ -429,6 +429,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   int *s_off = reinterpret_cast<int *>(s_dyn + kEWarps * sizeof(WarpShared));
 
   const int K = p.K;
+  chain_enter();
   const int n_rows = build_row_offsets(p.counts, p.B, p.rows_per_seq_max, s_off);   // the only barriers
   if (blockIdx.x == 0 && p.row_off)                  // the pruning kernel finds a sequence's rows with this
     for (int i = threadIdx.x; i <= p.B; i += kExpandThreads) p.row_off[i] = s_off[i];
@@ -577,9 +578,8 @@ cudaError_t prepare_expand_pass() {
 
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s) {
   const size_t smem = expand_dynamic_smem(p.B);
-  if (dtype == C2T_BF16) expand_pass_kernel<true><<<grid, kExpandThreads, smem, s>>>(p);
-  else expand_pass_kernel<false><<<grid, kExpandThreads, smem, s>>>(p);
-  return cudaGetLastError();
+  if (dtype == C2T_BF16) return launch_chained(expand_pass_kernel<true>, dim3(grid), dim3(kExpandThreads), smem, s, p);
+  return launch_chained(expand_pass_kernel<false>, dim3(grid), dim3(kExpandThreads), smem, s, p);
 }
 
 }  // namespace c2t

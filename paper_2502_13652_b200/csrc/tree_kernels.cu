@@ -43,6 +43,7 @@ __device__ int block_exclusive_scan(int v, int *s_warp /*[kTreeWarps+1]*/, int *
 }
 
 __global__ void begin_step_kernel(TreeState t, const int32_t *root_tok, const int32_t *prefix_len) {
+  chain_enter();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= t.B) return;
   const size_t o = (size_t)b * t.cap;
@@ -94,6 +95,19 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = t.K, F = t.F;
   const int cur = level & 1, nxt = cur ^ 1;
+  chain_release();
+  // the classifier's weights were written at init, not by the chain: they are staged while the
+  // expand pass may still be finishing
+  if (tid == 0) s_misc[1] = 0;                    // survivors of the first pruning
+  if (t.classifier == C2T_CLS_MLP) {
+    for (int i = tid; i < 3 * t.hidden; i += kTreeThreads) s_w[i] = t.w1[i];
+    for (int i = tid; i < t.hidden; i += kTreeThreads) {
+      s_w[3 * C2T_MAX_HIDDEN + i] = t.b1[i];
+      s_w[4 * C2T_MAX_HIDDEN + i] = t.w2[i];
+    }
+    if (tid == 0) s_w[5 * C2T_MAX_HIDDEN] = t.b2[0];
+  }
+  chain_wait();
   int n = t.frontier_n[cur][b];
   const int row_off = t.row_off_draft[b];         // rows of earlier sequences in the expand pass
   const PassInfo info = *t.info_draft;            // (loads issued together with the one above)
@@ -107,15 +121,6 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
       if (out.count) out.count[b] = 0;
     }
     return;
-  }
-  if (tid == 0) s_misc[1] = 0;                    // survivors of the first pruning
-  if (t.classifier == C2T_CLS_MLP) {
-    for (int i = tid; i < 3 * t.hidden; i += kTreeThreads) s_w[i] = t.w1[i];
-    for (int i = tid; i < t.hidden; i += kTreeThreads) {
-      s_w[3 * C2T_MAX_HIDDEN + i] = t.b1[i];
-      s_w[4 * C2T_MAX_HIDDEN + i] = t.w2[i];
-    }
-    if (tid == 0) s_w[5 * C2T_MAX_HIDDEN] = t.b2[0];
   }
   __syncthreads();
 
@@ -362,6 +367,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
 // is closed under "parent of".
 __global__ void __launch_bounds__(kTreeThreads) final_prune_kernel(TreeState t) {
   __shared__ int s_scan[kTreeWarps + 1];
+  chain_enter();
   const int b = blockIdx.x, tid = threadIdx.x;
   int n = t.tree_n[b];
   n = n > t.cap ? t.cap : n;
@@ -416,6 +422,7 @@ __global__ void __launch_bounds__(kTreeThreads) final_prune_kernel(TreeState t) 
 __global__ void __launch_bounds__(kTreeThreads) build_verify_kernel(TreeState t, c2t_verify out) {
   __shared__ int s_has_child[C2T_MAX_BUDGET > C2T_MAX_TREE ? C2T_MAX_BUDGET : C2T_MAX_TREE];
   __shared__ int s_scan[kTreeWarps + 1];
+  chain_enter();
   const int b = blockIdx.x, tid = threadIdx.x;
   const int n = t.final_n[b], Nw = t.Nw, W = t.W, width = t.D + 1;
   const size_t fb = (size_t)b * Nw;
@@ -470,6 +477,7 @@ __global__ void __launch_bounds__(kTreeThreads) build_verify_kernel(TreeState t,
 
 __global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, c2t_accept_out out) {
   __shared__ int s_misc[1];
+  chain_enter();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = t.final_n[b], Nw = t.Nw, width = t.D + 1;
   const size_t fb = (size_t)b * Nw;
@@ -576,6 +584,7 @@ constexpr int kWalkThreads = 1024;
 
 __global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState t, int round, c2t_accept_out out) {
   __shared__ int s_warp[kWalkThreads / 32 + 1];
+  chain_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int Nw = t.Nw, width = t.D + 1;
   const PassInfo info = *t.info_target;
@@ -670,40 +679,34 @@ cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_acce
   c2t_accept_out o;
   memset(&o, 0, sizeof o);
   if (out) o = *out;
-  lazy_walk_round_kernel<<<1, kWalkThreads, 0, s>>>(t, round, o);
-  return cudaGetLastError();
+  return launch_chained(lazy_walk_round_kernel, dim3(1), dim3(kWalkThreads), 0, s, t, round, o);
 }
 
 cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
                               cudaStream_t s) {
-  begin_step_kernel<<<(t.B + 127) / 128, 128, 0, s>>>(t, root_tok, prefix_len);
-  return cudaGetLastError();
+  return launch_chained(begin_step_kernel, dim3((t.B + 127) / 128), dim3(128), 0, s, t, root_tok, prefix_len);
 }
 
 cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s) {
   c2t_frontier o = {nullptr, nullptr, nullptr, nullptr};
   if (out) o = *out;
-  prune_level_kernel<<<t.B, kTreeThreads, 0, s>>>(t, level, o);
-  return cudaGetLastError();
+  return launch_chained(prune_level_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, level, o);
 }
 
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s) {
-  final_prune_kernel<<<t.B, kTreeThreads, 0, s>>>(t);
-  return cudaGetLastError();
+  return launch_chained(final_prune_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t);
 }
 
 cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s) {
   c2t_verify o = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   if (out) o = *out;
-  build_verify_kernel<<<t.B, kTreeThreads, 0, s>>>(t, o);
-  return cudaGetLastError();
+  return launch_chained(build_verify_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, o);
 }
 
 cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s) {
   c2t_accept_out o = {nullptr, nullptr, nullptr};
   if (out) o = *out;
-  accept_walk_kernel<<<t.B, kTreeThreads, 0, s>>>(t, o);
-  return cudaGetLastError();
+  return launch_chained(accept_walk_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, o);
 }
 
 }  // namespace c2t
