@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one expand_pass_kernel launch at this workload, from the ncu capture summarised in
 # profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  Set to
 # None when the kernel changes until the counters are taken again.
-EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.52e6}
+EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.09e6}
 
 
 def measured_hbm_peak():
@@ -354,6 +354,10 @@ def run_cuda(args) -> None:
             dist.destroy_process_group()
         return
 
+    # ---- the same expand kernel on fp32 logits (twice the bytes per element, the same arithmetic per element):
+    # reported beside the bf16 figure to show which side of the kernel the bytes-per-element ratio puts the bound on
+    fp32_level = expand_full_level_fp32(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream)
+
     # ---- roofline of the dominant kernel (the per-level vocabulary pass)
     peak, peak_kind = measured_hbm_peak()
     bytes_per_launch = sum(rows_per_level) * V * eb / D
@@ -407,12 +411,47 @@ def run_cuda(args) -> None:
                      "bytes_per_launch": bytes_per_launch,
                      "avg_launch_us": avg_launch_s * 1e6,
                      "full_level_rows": full_rows, "full_level_gbs": full_level_gbs,
-                     "frac_of_8000": achieved / 8000.0},
+                     "frac_of_8000": achieved / 8000.0,
+                     "fp32_logits_full_level": None if fp32_level is None else dict(
+                         fp32_level, frac=fp32_level["gbs"] / peak)},
         "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
     }
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def expand_full_level_fp32(c2t, dev, weights, root, prefix, stream, reps: int = 20):
+    """Times expand_pass_kernel<fp32> on full levels of the workload with fp32 logits (levels 1-3, three distinct
+    buffers of 328 MB, so every launch reads from DRAM).  Returns None if the frontier does not fill."""
+    w = WORKLOAD
+    B, V, K, F, N = w["B"], w["V"], w["K"], w["F"], w["N"]
+    levels = 4
+    w1, b1, w2, b2 = weights
+    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32, max_depth=levels, topk=K, frontier_cap=F, budget=N,
+                     threshold=w["beta"], hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
+    ctx = c2t.Context(cfg)
+    draft = [c2t_inputs.draft_logits(B, F, V, 0, l, torch.float32, device=dev) for l in range(levels)]
+    rows = []
+    ms = []
+    for rep in range(reps + 3):
+        ctx.c2t_begin_step(root, prefix, stream)
+        for l in range(levels):
+            if rep == 0:
+                rows.append(int(ctx.c2t_get_view()["frontier_n"].sum().item()))
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            ctx.c2t_expand_level(l, draft[l], stream)
+            b.record()
+            ctx.c2t_prune(l, stream)
+            if rep >= 3 and l >= 1:
+                ms.append((a, b))
+    torch.cuda.synchronize()
+    if min(rows[1:]) != B * F:
+        return None
+    us = sum(a.elapsed_time(b) for a, b in ms) / len(ms) * 1e3
+    nbytes = B * F * V * 4
+    return {"rows": B * F, "bytes": nbytes, "us": us, "gbs": nbytes / (us * 1e-6) / 1e9}
 
 
 def run_profile(args) -> None:
