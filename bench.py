@@ -358,6 +358,9 @@ def run_cuda(args) -> None:
     # reported beside the bf16 figure to show which side of the kernel the bytes-per-element ratio puts the bound on
     fp32_level = expand_full_level_fp32(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream)
 
+    # ---- the single-sequence configuration (latency-bound), timed per decode step; one GPU only
+    single_seq = single_sequence_latency(c2t, dev, default_stream) if world == 1 else None
+
     # ---- roofline of the dominant kernel (the per-level vocabulary pass)
     peak, peak_kind = measured_hbm_peak()
     bytes_per_launch = sum(rows_per_level) * V * eb / D
@@ -401,6 +404,7 @@ def run_cuda(args) -> None:
         "lazy_accept": {"us_per_step": lazy_ms_per_step * 1e3,
                         "value": whole_job_levels_per_second(world, B, D, lazy_ms_per_step), "unit": UNIT,
                         "note": "c2t_accept_lazy: accept_len+1 target rows per sequence instead of all final nodes"},
+        "single_sequence": single_seq,
         "clocks": clocks,
         "e2e": {"value": whole_job_levels_per_second(world, B, D, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -452,6 +456,72 @@ def expand_full_level_fp32(c2t, dev, weights, root, prefix, stream, reps: int = 
     us = sum(a.elapsed_time(b) for a, b in ms) / len(ms) * 1e3
     nbytes = B * F * V * 4
     return {"rows": B * F, "bytes": nbytes, "us": us, "gbs": nbytes / (us * 1e-6) / 1e9}
+
+
+def single_sequence_latency(c2t, dev, stream, steps: int = 60, sets: int = 4):
+    """The single-stream case: B=1, V=128256, bf16, D=10, K=8, F=16, N=80, thresholds 0.3 / 0.5 / 0.7; µs per decode
+    step.  One step's logits (61 MB) would stay in L2, so the steps rotate over `sets` input sets (246 MB)."""
+    B, V, D, K, F, N, hidden = 1, 128256, 10, 8, 16, 80, 16
+    w1, b1, w2, b2 = make_weights(hidden)
+    out = {"workload": "B=1, V=128256, bf16, depth 10, top-k 8, frontier cap 16, budget 80, MLP hidden 16",
+           "l2": f"steps rotate over {sets} input sets (246 MB, larger than L2)", "us_per_step": {}, "us_per_step_graph_replay": {}, "rows_per_step": {}}
+    inputs = None
+    for beta in (0.3, 0.5, 0.7):
+        cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.BF16, max_depth=D, topk=K, frontier_cap=F, budget=N,
+                         threshold=beta, hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
+        ctx = c2t.Context(cfg)
+        if inputs is None:
+            inputs = []
+            for k in range(sets):
+                draft = [c2t_inputs.draft_logits(B, F, V, k, l, torch.bfloat16, device=dev) for l in range(D)]
+                target = c2t_inputs.target_logits(B, ctx.Nw, V, k, torch.bfloat16, device=dev)
+                inputs.append((draft, target, c2t_inputs.root_tokens(B, V, k).to(dev),
+                               c2t_inputs.prefix_lengths(B).to(dev)))
+        rows = 0
+        ctx.c2t_begin_step(inputs[0][2], inputs[0][3], stream)
+        for l in range(D):
+            rows += int(ctx.c2t_get_view()["frontier_n"].sum().item())
+            ctx.c2t_expand_level(l, inputs[0][0][l], stream)
+            ctx.c2t_prune(l, stream)
+        for i in range(4):
+            ctx.decode_step(*inputs[i % sets], stream=stream)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(steps):
+            ctx.decode_step(*inputs[i % sets], stream=stream)
+        b.record()
+        torch.cuda.synchronize()
+        out["us_per_step"][str(beta)] = a.elapsed_time(b) / steps * 1e3
+        out["rows_per_step"][str(beta)] = rows
+        # the same steps replayed from CUDA graphs (one per input set): 24 launches of a few microseconds each are
+        # bounded by the host's launch calls otherwise
+        try:
+            side = torch.cuda.Stream(device=dev)
+            graphs = []
+            for k in range(sets):
+                with torch.cuda.stream(side):
+                    ctx.decode_step(*inputs[k], stream=side.cuda_stream)
+                torch.cuda.synchronize()
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=side):
+                    ctx.decode_step(*inputs[k], stream=torch.cuda.current_stream().cuda_stream)
+                graphs.append(gr)
+            for i in range(4):
+                graphs[i % sets].replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(steps):
+                graphs[i % sets].replay()
+            b.record()
+            torch.cuda.synchronize()
+            out["us_per_step_graph_replay"][str(beta)] = a.elapsed_time(b) / steps * 1e3
+            del graphs
+        except RuntimeError as exc:
+            print(f"bench.py: CUDA graph replay of the single-sequence case skipped: {exc}", file=sys.stderr)
+        ctx.close()
+    return out
 
 
 def run_profile(args) -> None:

@@ -11,3 +11,4 @@ from .binding import (  # noqa: F401
     OK, EINVAL, EALIGN, ERANGE, EORDER, ECUDA,
     ST_NAN_LOGIT, ST_POSINF_LOGIT, ST_ALL_NEGINF, ST_TREE_OVERFLOW,
 )
+from .weights import save_classifier, load_classifier  # noqa: F401,E402

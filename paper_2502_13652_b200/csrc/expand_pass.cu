@@ -14,8 +14,8 @@
 // three smaller ones: the warps of an older CTA are served first, and its work would end early.)
 //
 // Data movement.  A warp works on groups of 128 consecutive vectors (2 KB), four per lane, 32
-// apart.  Each lane owns 4 x 16 bytes in each of two shared-memory slots and fills them with
-// cp.async: while group n is in registers, groups n+1 and n+2 are in flight, across segment
+// apart.  Each lane owns 4 x 16 bytes in each of kRingSlots shared-memory slots and fills them with
+// cp.async: while group n is in registers, groups n+1 .. n+kRingSlots are in flight, across segment
 // boundaries too.  A lane reads back only what it copied itself, so the only wait is on its own
 // copies (cp.async.wait_group).
 //
@@ -45,13 +45,14 @@ namespace {
 
 constexpr int kEWarps = kExpandThreads / 32;
 constexpr int kGroupVecs = 128;                       // vectors of one group of a warp
+constexpr int kRingSlots = 2;                         // groups in flight per warp behind the one in registers (3 measured 3 % slower)
 constexpr int kDrainAt = 12;                          // queued vectors that trigger a drain: early drains keep the filter tight
 constexpr int kQueueCap = kDrainAt + kGroupVecs;      // a whole group always fits behind kDrainAt vectors
 
 // What one warp owns in shared memory.
 constexpr int kPool = 64;                             // keys ranked at a time (the K kept ones and up to 32 + 32 - K new)
 struct WarpShared {
-  uint4 ring[2][kGroupVecs];
+  uint4 ring[kRingSlots][kGroupVecs];
   uint4 qdata[kQueueCap];
   int qindex[kQueueCap];
   unsigned long long pool[kPool];      // [0, K): the K largest keys so far, sorted (0 = none); behind them the new ones
@@ -187,6 +188,7 @@ __device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void *gmem_
   asm volatile("cp.async.cg.shared.global [%0 + %2], [%1 + %2], 16;" ::"r"(smem_dst), "l"(gmem_src), "n"(OFF) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ unsigned next_slot(unsigned slot) { return slot + 1 == kRingSlots ? 0u : slot + 1; }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -257,7 +259,7 @@ __device__ __noinline__ float2 segment_warmup(int K, Group g, int vt, int v1, in
       if (vm == vm) lmax = fmaxf(lmax, vm);
     }
   }
-  cp_async_wait<1>();                      // the group after this one (all but the newest request)
+  cp_async_wait<kRingSlots - 1>();         // the group after this one (the oldest request)
   const int lim = v1 < v_full ? v1 : v_full;
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
@@ -455,14 +457,15 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   const size_t esz = BF16 ? 2 : 4;
   GroupCursor cur(start, end, vpr, p, s_off, esz);   // the group being worked on
   GroupCursor pre = cur;                             // the group being requested, two ahead
-  prefetch_group(pre, ws->ring[0], v_full, lane);
-  pre.advance(p, s_off, esz);
-  prefetch_group(pre, ws->ring[1], v_full, lane);
-  pre.advance(p, s_off, esz);
-  unsigned n = 0;                                    // index of the current group: its ring slot is n & 1
+#pragma unroll
+  for (int i = 0; i < kRingSlots; ++i) {
+    prefetch_group(pre, ws->ring[i], v_full, lane);
+    pre.advance(p, s_off, esz);
+  }
+  unsigned n = 0;                                    // ring slot of the current group
 
   Group g;
-  cp_async_wait<1>();
+  cp_async_wait<kRingSlots - 1>();
   take_group<BF16>(g, cur, ws->ring[0], v_full, p.V, lane);
   prefetch_group(pre, ws->ring[0], v_full, lane);
   pre.advance(p, s_off, esz);
@@ -473,7 +476,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   for (;;) {
     const Segment seg = cur.seg;
     if (fresh) {
-      const float2 w = segment_warmup<BF16>(K, g, cur.tv0 + lane, seg.v1, v_full, ws->ring[(n + 1) & 1u]);
+      const float2 w = segment_warmup<BF16>(K, g, cur.tv0 + lane, seg.v1, v_full, ws->ring[next_slot(n)]);
       st.acc.S0 = st.acc.S1 = st.acc.U0 = st.acc.U1 = 0.f;
       st.thr = w.x;
       st.m = w.y;
@@ -483,19 +486,19 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       fresh = false;
     }
     // ---- the inside of a segment: this group, the next one (in the ring) and the one to be
-    // requested (three ahead) are whole groups of this segment, so nothing needs checking
+    // requested (kRingSlots + 1 ahead) are whole groups of this segment, so nothing needs checking
     if (pre.valid && pre.seg.a == seg.a) {
       const int lim = seg.v1 < v_full ? seg.v1 : v_full;
-      const int k = (lim - cur.tv0) / kGroupVecs - 3;
+      const int k = (lim - cur.tv0) / kGroupVecs - (kRingSlots + 1);
       if (k > 0) {
         const uint4 *src = reinterpret_cast<const uint4 *>(seg.row) + pre.tv0 + lane;
         int vt = cur.tv0 + lane;
         for (int i = 0; i < k; ++i) {
           process_group<BF16, true>(ws, g, st, vt, 0, lt_mask);
-          ++n;
+          n = next_slot(n);
           vt += kGroupVecs;
-          cp_async_wait<1>();
-          uint4 *slot = ws->ring[n & 1u];
+          cp_async_wait<kRingSlots - 1>();
+          uint4 *slot = ws->ring[n];
 #pragma unroll
           for (int u = 0; u < 4; ++u) g.q[u] = slot[lane + u * 32];
 #pragma unroll
@@ -519,10 +522,10 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
     process_group<BF16, false>(ws, g, st, vt, seg.v1, lt_mask);
     const bool last = cur.last_of_segment();
     cur.advance(p, s_off, esz);
-    ++n;
+    n = next_slot(n);
     if (cur.valid) {                                 // next group (of this or of the next segment) into registers
-      cp_async_wait<1>();
-      uint4 *slot = ws->ring[n & 1u];
+      cp_async_wait<kRingSlots - 1>();
+      uint4 *slot = ws->ring[n];
       take_group<BF16>(g, cur, slot, v_full, p.V, lane);
       prefetch_group(pre, slot, v_full, lane);
       pre.advance(p, s_off, esz);

@@ -299,6 +299,47 @@ def test_results_are_reproducible():
     ctx.close()
 
 
+def test_back_to_back_steps_equal_isolated_steps():
+    """Steps queued without any host synchronisation give what the same steps give one at a time.
+    The kernels of a step are launched so that each may be placed on the SMs while its predecessor is
+    still finishing and waits for it before its first access to memory; a kernel that ran ahead of
+    that wait would read the other input set's frontier or partial records here."""
+    B, V, D, K, F, N = 8, 32000, 5, 10, 10, 40
+    _, gcfg = make_configs(B, V, D, K, F, N, 0.5, torch.bfloat16)
+    Nw = c2t.c2t_final_width(gcfg)
+    sets = []
+    for step in (0, 1):
+        draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, torch.bfloat16, step=step)
+        sets.append(([t.cuda() for t in draft], target.cuda(), root.cuda(), prefix.cuda()))
+    ctx = c2t.Context(gcfg)
+
+    def snapshot():                                      # device-side copies in stream order, no synchronisation
+        v = ctx.c2t_get_view()
+        n = v["tree_n"].clone()
+        live = torch.arange(ctx.cap, device="cuda")[None, :] < n[:, None]
+        return [n, torch.where(live, v["tree_token"], 0), torch.where(live, v["tree_parent"], 0),
+                torch.where(live, v["tree_logP"], 0.0), torch.where(live, v["tree_C"], 0.0),
+                ctx.verify["mask_bits"].clone(), ctx.verify["retrieve"].clone(),
+                ctx.accepted["accept_len"].clone(), ctx.accepted["path"].clone(), ctx.accepted["next_token"].clone()]
+
+    alone = []
+    for inp in sets:
+        ctx.decode_step(*inp)
+        torch.cuda.synchronize()
+        alone.append(snapshot())
+        torch.cuda.synchronize()
+    assert not all(torch.equal(a, b) for a, b in zip(alone[0], alone[1]))     # the two sets do differ
+    queued = []
+    for i in range(24):                                  # no synchronisation inside this loop
+        ctx.decode_step(*sets[i & 1])
+        queued.append(snapshot())
+    torch.cuda.synchronize()
+    for i, snap in enumerate(queued):
+        for a, b in zip(alone[i & 1], snap):
+            assert torch.equal(a, b), i
+    ctx.close()
+
+
 @pytest.mark.parametrize("dtype,V,M", [(torch.bfloat16, 32000, 1000), (torch.float32, 32000, 1000),
                                        (torch.bfloat16, 5000, 100), (torch.float32, 4096, 5),
                                        (torch.bfloat16, 3000, 3000), (torch.float32, 3000, 7000)])

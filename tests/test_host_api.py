@@ -127,3 +127,22 @@ def test_struct_layouts_match_the_header():
             for part in decl.split(","):
                 names.append(re.findall(r"([A-Za-z_0-9]+)\s*$", part.strip())[0])
         assert names == [n for n, _ in mirror._fields_], struct
+
+
+def test_classifier_weights_file_round_trip(tmp_path):
+    """save_classifier / load_classifier keep every float32 bit and refuse damaged files."""
+    import c2t_inputs
+    from paper_2502_13652_b200 import save_classifier, load_classifier
+    w = c2t_inputs.classifier_weights(48, seed=3)
+    path = str(tmp_path / "ffn.c2tw")
+    save_classifier(path, *w)
+    back = load_classifier(path)
+    for a, b in zip(w, back):
+        assert a.dtype == b.dtype == torch.float32 and a.shape == b.shape and torch.equal(a, b)
+    blob = open(path, "rb").read()
+    for bad in (blob[:-4], b"X" + blob[1:], blob + b"\0\0\0\0"):
+        open(path, "wb").write(bad)
+        with pytest.raises(ValueError):
+            load_classifier(path)
+    with pytest.raises(ValueError):
+        save_classifier(path, torch.zeros(65, 3), torch.zeros(65), torch.zeros(65), torch.zeros(1))
