@@ -44,7 +44,8 @@ namespace c2t {
 namespace {
 
 constexpr int kEWarps = kExpandThreads / 32;
-constexpr int kGroupVecs = 128;                       // vectors of one group of a warp
+constexpr int kVPL = kExpandVecPerLane;               // vectors of a group per lane, 32 apart
+constexpr int kGroupVecs = 32 * kVPL;                 // vectors of one group of a warp
 constexpr int kRingSlots = 2;                         // groups in flight per warp behind the one in registers (3 measured 3 % slower)
 constexpr int kDrainAt = 12;                          // queued vectors that trigger a drain: early drains keep the filter tight
 constexpr int kQueueCap = kDrainAt + kGroupVecs;      // a whole group always fits behind kDrainAt vectors
@@ -109,7 +110,7 @@ struct SegState {
 };
 
 struct Group {
-  uint4 q[4];
+  uint4 q[kVPL];
 };
 
 // ---------------------------------------------------------------- segments of a span
@@ -192,24 +193,32 @@ __device__ __forceinline__ unsigned next_slot(unsigned slot) { return slot + 1 =
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// the lane's kVPL copies of a whole group / of a group cut off at vector lim
+template <int U>
+struct LaneCopies {
+  static __device__ __forceinline__ void all(uint32_t dst, const uint4 *src) {
+    LaneCopies<U - 1>::all(dst, src);
+    cp_async_16<(U - 1) * 512>(dst, src);
+  }
+  static __device__ __forceinline__ void below(uint32_t dst, const uint4 *src, int vt, int lim) {
+    LaneCopies<U - 1>::below(dst, src, vt, lim);
+    if (vt + (U - 1) * 32 < lim) cp_async_16<(U - 1) * 512>(dst, src);
+  }
+};
+template <>
+struct LaneCopies<0> {
+  static __device__ __forceinline__ void all(uint32_t, const uint4 *) {}
+  static __device__ __forceinline__ void below(uint32_t, const uint4 *, int, int) {}
+};
+
 // Requests the whole vectors of the cursor's group into the lane's places of a ring slot.
 __device__ __forceinline__ void prefetch_group(const GroupCursor &c, uint4 *slot, int v_full, int lane) {
   if (c.valid) {
     const int lim = c.seg.v1 < v_full ? c.seg.v1 : v_full;
     const uint4 *src = reinterpret_cast<const uint4 *>(c.seg.row) + c.tv0 + lane;
     const uint32_t dst = (uint32_t)__cvta_generic_to_shared(slot + lane);
-    if (c.tv0 + kGroupVecs <= lim) {
-      cp_async_16<0>(dst, src);
-      cp_async_16<512>(dst, src);
-      cp_async_16<1024>(dst, src);
-      cp_async_16<1536>(dst, src);
-    } else {
-      const int vt = c.tv0 + lane;
-      if (vt < lim) cp_async_16<0>(dst, src);
-      if (vt + 32 < lim) cp_async_16<512>(dst, src);
-      if (vt + 64 < lim) cp_async_16<1024>(dst, src);
-      if (vt + 96 < lim) cp_async_16<1536>(dst, src);
-    }
+    if (c.tv0 + kGroupVecs <= lim) LaneCopies<kVPL>::all(dst, src);
+    else LaneCopies<kVPL>::below(dst, src, c.tv0 + lane, lim);
   }
   cp_async_commit();
 }
@@ -225,17 +234,17 @@ __device__ __forceinline__ void take_group(Group &g, const GroupCursor &c, const
   const int vt = c.tv0 + lane;
   if (c.tv0 + kGroupVecs <= (c.seg.v1 < v_full ? c.seg.v1 : v_full)) {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) g.q[u] = slot[lane + u * 32];
+    for (int u = 0; u < kVPL; ++u) g.q[u] = slot[lane + u * 32];
   } else {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kVPL; ++u) {
       const int v = vt + u * 32;
       g.q[u] = make_uint4(lo, lo, lo, lo);
       if (v < c.seg.v1) g.q[u] = v < v_full ? slot[lane + u * 32] : VT::load(c.seg.row, v, v_full, V);
     }
   }
 #pragma unroll
-  for (int u = 0; u < 4; ++u) VT::clamp(g.q[u]);
+  for (int u = 0; u < kVPL; ++u) VT::clamp(g.q[u]);
 }
 
 // ---------------------------------------------------------------- start of a segment
@@ -253,7 +262,7 @@ __device__ __noinline__ float2 segment_warmup(int K, Group g, int vt, int v1, in
   const int lane = threadIdx.x & 31;
   float lmax = -INFINITY;
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
+  for (int u = 0; u < kVPL; ++u) {
     if (vt + u * 32 < v1) {
       const float vm = VT::vmax(g.q[u]);
       if (vm == vm) lmax = fmaxf(lmax, vm);
@@ -262,7 +271,7 @@ __device__ __noinline__ float2 segment_warmup(int K, Group g, int vt, int v1, in
   cp_async_wait<kRingSlots - 1>();         // the group after this one (the oldest request)
   const int lim = v1 < v_full ? v1 : v_full;
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
+  for (int u = 0; u < kVPL; ++u) {
     if (vt + kGroupVecs + u * 32 < lim) {  // same segment, whole vector: it is in the ring
       uint4 q = next_slot[lane + u * 32];
       VT::clamp(q);
@@ -379,25 +388,28 @@ template <bool BF16, bool WHOLE>
 __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, SegState &st, int vt, int v1,
                                               unsigned lt_mask) {
   using VT = Vec<BF16>;
-  float vm[4];
+  float vm[kVPL];
 #pragma unroll
-  for (int u = 0; u < 4; ++u) vm[u] = VT::vmax(g.q[u]);
-  const bool any_hit = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])) >= st.thr;
+  for (int u = 0; u < kVPL; ++u) vm[u] = VT::vmax(g.q[u]);
+  float gm = vm[0];
+#pragma unroll
+  for (int u = 1; u < kVPL; ++u) gm = fmaxf(gm, vm[u]);
+  const bool any_hit = gm >= st.thr;
   if (!__any_sync(kFull, any_hit)) {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) acc_vector<BF16>(st.acc, g.q[u], kLog2e, st.c);
+    for (int u = 0; u < kVPL; ++u) acc_vector<BF16>(st.acc, g.q[u], kLog2e, st.c);
   } else {
     // The sums still run over all four vectors in one straight line; a vector that goes to the
     // queue is left out by t = 0 x - 200 (2^-200 flushes to zero and 0 * -200 adds nothing to U).
-    bool hit[4];
-    unsigned mask[4];
+    bool hit[kVPL];
+    unsigned mask[kVPL];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kVPL; ++u) {
       hit[u] = vm[u] >= st.thr && (WHOLE || vt + u * 32 < v1);
       mask[u] = __ballot_sync(kFull, hit[u]);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kVPL; ++u) {
       if (hit[u]) {
         const int pos = st.qn + __popc(mask[u] & lt_mask);
         ws->qdata[pos] = g.q[u];
@@ -406,7 +418,7 @@ __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, Se
       st.qn += __popc(mask[u]);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < kVPL; ++u)
       acc_vector<BF16>(st.acc, g.q[u], hit[u] ? 0.f : kLog2e, hit[u] ? -200.f : st.c);
   }
 }
@@ -500,14 +512,11 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
           cp_async_wait<kRingSlots - 1>();
           uint4 *slot = ws->ring[n];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) g.q[u] = slot[lane + u * 32];
+          for (int u = 0; u < kVPL; ++u) g.q[u] = slot[lane + u * 32];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) VT::clamp(g.q[u]);
+          for (int u = 0; u < kVPL; ++u) VT::clamp(g.q[u]);
           const uint32_t dst = (uint32_t)__cvta_generic_to_shared(slot + lane);
-          cp_async_16<0>(dst, src);
-          cp_async_16<512>(dst, src);
-          cp_async_16<1024>(dst, src);
-          cp_async_16<1536>(dst, src);
+          LaneCopies<kVPL>::all(dst, src);
           cp_async_commit();
           src += kGroupVecs;
           if (st.qn > kDrainAt) drain_into<BF16>(ws, st, K);
