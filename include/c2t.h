@@ -67,6 +67,7 @@ typedef enum { C2T_ADD_FRONTIER = 0, C2T_ADD_ALL_SURVIVORS = 1 } c2t_tree_add;
 #define C2T_MAX_DEPTH     32
 #define C2T_MAX_BUDGET    1024
 #define C2T_MAX_TREE      8192   /* nodes per sequence before the Top-N rerank */
+#define C2T_MAX_SHARDS    32     /* vocabulary shards merged by c2t_prune_gathered */
 
 /* per-sequence status bits */
 #define C2T_ST_NAN_LOGIT     1u
@@ -192,6 +193,67 @@ int c2t_build_verify(c2t_ctx *ctx, const c2t_verify *out, void *stream);
  * unknown out_dtype.
  */
 int c2t_dense_mask(c2t_ctx *ctx, void *out_dev, int32_t out_dtype, int64_t kv_len, void *stream);
+
+/*
+ * Vocabulary-parallel levels.  When the draft model's output layer is sharded over the vocabulary,
+ * each GPU holds the logits of a contiguous token range [vocab_begin, vocab_begin + vocab_count) of
+ * every frontier row.  A level is then built in three calls instead of two:
+ *
+ *   c2t_expand_level_shard   the vocabulary pass of c2t_expand_level over this range only;
+ *   c2t_export_row_records   one c2t_row_record per active row: the range's maximum, its softmax and
+ *                            entropy sums relative to that maximum, its K largest logits with GLOBAL
+ *                            token ids (the quantities of Sec. 4.2.1, Eq. 2 and Sec. 4.2.2 restricted
+ *                            to the range);
+ *   (the caller all-gathers the records of all ranges: [n_shards, B, F] records, shard-major, in
+ *    ascending order of vocab_begin; 288 bytes per row and shard)
+ *   c2t_prune_gathered       c2t_prune(level) with the rows' sums and candidates merged from the
+ *                            gathered records instead of from this context's own pass: the maxima are
+ *                            aligned (sums rescaled by e^(M_shard - M)), a shard's own maximum rejoins
+ *                            the sums unless it is the row's, and the K best of the shards' lists are
+ *                            taken under the usual order (logit descending, token id ascending).
+ *
+ * The results are those of c2t_expand_level + c2t_prune on the full rows up to fp64 rounding of the
+ * merge.  A range whose elements are all -inf contributes nothing; NaN and +inf set the status bits of
+ * the sequence as usual.  Ranges must be disjoint, cover [0, V), and every vocab_begin must keep the
+ * shard's rows 16-byte aligned.  The truncated entropy of Eq. 3 (entropy_top_m) is not available in
+ * this mode (C2T_EINVAL).
+ */
+typedef struct {
+  double  M;                     /* largest logit of the range (its best key's value)              */
+  double  S;                     /* sum over the range's OTHER elements of e^(x - M)                */
+  double  T;                     /* sum over the range's other elements of e^(x - M) (x - M)        */
+  int32_t n;                     /* entries of tok / x that are valid (at most K)                   */
+  uint32_t fault;                /* C2T_ST_* bits of this range of this row                         */
+  int32_t tok[C2T_MAX_TOPK];     /* global token ids of the range's largest logits, best first      */
+  float   x[C2T_MAX_TOPK];       /* those logits                                                    */
+} c2t_row_record;
+
+/*
+ * The vocabulary pass of level `level` over one token range (Sec. 4.2.1, Eq. 2, Sec. 4.2.2).
+ * logits_dev: [B, F, vocab_count] of cfg.dtype with the strides and alignment rules of
+ * c2t_expand_level (row_stride >= vocab_count); 1 <= vocab_count <= V.  Same call order as
+ * c2t_expand_level; must be followed by c2t_export_row_records before anything else.
+ */
+int c2t_expand_level_shard(c2t_ctx *ctx, int level, const void *logits_dev, int64_t seq_stride,
+                           int64_t row_stride, int32_t vocab_count, void *stream);
+
+/*
+ * Writes the record of every active row (b, j) of the pass just run to records_dev[b * F + j]
+ * (device memory of the caller, B * F records; rows j >= the sequence's frontier size are not
+ * written).  vocab_begin is added to the token ids; vocab_begin + vocab_count <= V.
+ */
+int c2t_export_row_records(c2t_ctx *ctx, int level, int32_t vocab_begin, c2t_row_record *records_dev,
+                           void *stream);
+
+/*
+ * c2t_prune(level) from gathered records (Eq. 1, Eq. 4, Alg. 1's two prunings): records_dev is
+ * [n_shards, B, F], shard s of row (b, j) at (s * B + b) * F + j; 1 <= n_shards <= C2T_MAX_SHARDS.
+ * `level` must be the level whose records were exported; the next call is c2t_expand_level(_shard)
+ * of level + 1 or c2t_prune(C2T_FINAL).  Every rank that calls it with the same records builds the
+ * same tree.
+ */
+int c2t_prune_gathered(c2t_ctx *ctx, int level, const c2t_row_record *records_dev, int32_t n_shards,
+                       const c2t_frontier *out, void *stream);
 
 typedef struct {
   int32_t *accept_len;   /* [B]      tau of this step: accepted draft tokens, root excluded */

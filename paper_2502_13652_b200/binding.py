@@ -44,6 +44,18 @@ class c2t_frontier(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("count", "token", "node_id", "parent_slot")]
 
 
+MAX_TOPK = 32
+MAX_SHARDS = 32
+
+
+class c2t_row_record(C.Structure):
+    _fields_ = [("M", C.c_double), ("S", C.c_double), ("T", C.c_double), ("n", C.c_int32), ("fault", C.c_uint32),
+                ("tok", C.c_int32 * MAX_TOPK), ("x", C.c_float * MAX_TOPK)]
+
+
+ROW_RECORD_BYTES = C.sizeof(c2t_row_record)      # 288
+
+
 class c2t_verify(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("n_nodes", "tokens", "parents", "position_ids", "mask_bits",
                                           "retrieve", "n_leaves")]
@@ -102,6 +114,13 @@ def lib() -> C.CDLL:
         L.c2t_expand_level.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p]
         L.c2t_prune.restype = C.c_int
         L.c2t_prune.argtypes = [C.c_void_p, C.c_int, P(c2t_frontier), C.c_void_p]
+        L.c2t_expand_level_shard.restype = C.c_int
+        L.c2t_expand_level_shard.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
+                                             C.c_void_p]
+        L.c2t_export_row_records.restype = C.c_int
+        L.c2t_export_row_records.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_void_p]
+        L.c2t_prune_gathered.restype = C.c_int
+        L.c2t_prune_gathered.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int32, P(c2t_frontier), C.c_void_p]
         L.c2t_build_verify.restype = C.c_int
         L.c2t_build_verify.argtypes = [C.c_void_p, P(c2t_verify), C.c_void_p]
         L.c2t_accept.restype = C.c_int
@@ -289,6 +308,34 @@ class Context:
     def c2t_prune(self, level: int, stream=None, emit: bool = True) -> None:
         out = C.byref(self._frontier_c) if (emit and level != FINAL) else None
         _check(lib().c2t_prune(self._h, level, out, _stream(stream)), "c2t_prune")
+
+    def c2t_expand_level_shard(self, level: int, logits: torch.Tensor, stream=None) -> None:
+        """logits: [B, >=F, vocab_count] CUDA tensor of the configured dtype, last dimension contiguous (a slice of
+        wider rows is fine: the strides are the tensor's)."""
+        assert logits.is_cuda and logits.dtype == self.cfg.torch_dtype and logits.dim() == 3
+        assert logits.shape[0] == self.B and logits.stride(2) == 1
+        _check(lib().c2t_expand_level_shard(self._h, level, logits.data_ptr(), logits.stride(0), logits.stride(1),
+                                            logits.shape[2], _stream(stream)), "c2t_expand_level_shard")
+
+    def new_row_records(self, n_shards: int = 1) -> torch.Tensor:
+        """Device buffer for [n_shards, B, F] row records, as bytes (see `c2t_row_record`)."""
+        return torch.zeros((n_shards, self.B, self.F, ROW_RECORD_BYTES), dtype=torch.uint8,
+                           device=self.workspace.device)
+
+    def c2t_export_row_records(self, level: int, vocab_begin: int, records: torch.Tensor, stream=None) -> None:
+        """records: [B, F, ROW_RECORD_BYTES] uint8 CUDA tensor, contiguous (one shard's slot of `new_row_records`)."""
+        assert records.is_cuda and records.dtype == torch.uint8 and records.is_contiguous()
+        assert records.numel() == self.B * self.F * ROW_RECORD_BYTES
+        _check(lib().c2t_export_row_records(self._h, level, vocab_begin, records.data_ptr(), _stream(stream)),
+               "c2t_export_row_records")
+
+    def c2t_prune_gathered(self, level: int, records: torch.Tensor, stream=None, emit: bool = True) -> None:
+        """records: [n_shards, B, F, ROW_RECORD_BYTES] uint8 CUDA tensor, shards in ascending token order."""
+        assert records.is_cuda and records.dtype == torch.uint8 and records.is_contiguous() and records.dim() == 4
+        assert records.shape[1:] == (self.B, self.F, ROW_RECORD_BYTES)
+        out = C.byref(self._frontier_c) if emit else None
+        _check(lib().c2t_prune_gathered(self._h, level, records.data_ptr(), records.shape[0], out, _stream(stream)),
+               "c2t_prune_gathered")
 
     def c2t_build_verify(self, stream=None) -> None:
         _check(lib().c2t_build_verify(self._h, C.byref(self._verify_c), _stream(stream)), "c2t_build_verify")

@@ -13,6 +13,8 @@ struct c2t_ctx {
   int grid_expand;       // CTAs of the expand pass
   int next_level;        // level the next c2t_expand_level must carry
   int expanded;          // 1 after expand_level(next_level), before its prune
+  int shard_expanded;    // 1 after expand_level_shard(next_level), before its export
+  int shard_vocab;       // tokens of that shard
   int finalized;         // 1 after c2t_prune(C2T_FINAL)
   int started;
   int64_t launches;
@@ -223,6 +225,7 @@ int c2t_begin_step(c2t_ctx *ctx, const int32_t *root_tok_dev, const int32_t *pre
   ctx->launches += 1;
   ctx->next_level = 0;
   ctx->expanded = 0;
+  ctx->shard_expanded = 0;
   ctx->finalized = 0;
   ctx->started = 1;
   return C2T_OK;
@@ -231,7 +234,7 @@ int c2t_begin_step(c2t_ctx *ctx, const int32_t *root_tok_dev, const int32_t *pre
 int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t seq_stride,
                      int64_t row_stride, void *stream) {
   if (!ctx || !logits_dev) return C2T_EINVAL;
-  if (!ctx->started || ctx->finalized || ctx->expanded || level != ctx->next_level ||
+  if (!ctx->started || ctx->finalized || ctx->expanded || ctx->shard_expanded || level != ctx->next_level ||
       level >= ctx->cfg.max_depth)
     return C2T_EORDER;
   if (seq_stride < 0 || row_stride < ctx->cfg.vocab) return C2T_EINVAL;
@@ -271,9 +274,65 @@ int c2t_prune(c2t_ctx *ctx, int level, const c2t_frontier *out, void *stream) {
     return C2T_OK;
   }
   if (!ctx->expanded || level != ctx->next_level) return C2T_EORDER;
-  if (launch_prune_level(ctx->t, level, out, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
+  if (launch_prune_level(ctx->t, level, out, nullptr, 0, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
   ctx->launches += 1;
   ctx->expanded = 0;
+  ctx->next_level = level + 1;
+  return C2T_OK;
+}
+
+int c2t_expand_level_shard(c2t_ctx *ctx, int level, const void *logits_dev, int64_t seq_stride,
+                           int64_t row_stride, int32_t vocab_count, void *stream) {
+  if (!ctx || !logits_dev) return C2T_EINVAL;
+  if (!ctx->started || ctx->finalized || ctx->expanded || ctx->shard_expanded || level != ctx->next_level ||
+      level >= ctx->cfg.max_depth)
+    return C2T_EORDER;
+  if (vocab_count < 1 || vocab_count > ctx->cfg.vocab || seq_stride < 0 || row_stride < vocab_count) return C2T_EINVAL;
+  if (ctx->t.entropy_top_m > 0 && ctx->t.entropy_top_m < ctx->t.V) return C2T_EINVAL;   // Eq. 3 needs whole rows
+  if (!aligned16(logits_dev) || (seq_stride * ctx->elem_bytes) % 16 || (row_stride * ctx->elem_bytes) % 16)
+    return C2T_EALIGN;
+  const TreeState &t = ctx->t;
+  PassParams p;
+  memset(&p, 0, sizeof p);
+  p.logits = logits_dev; p.seq_stride = seq_stride; p.row_stride = row_stride;
+  p.V = vocab_count; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
+  p.counts = t.frontier_n[level & 1];
+  p.max_splits = t.max_splits;                    // sized for whole rows: enough for any part of one
+  p.info = t.info_draft;
+  p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
+  p.row_off = t.row_off_draft;
+  if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid_expand, (cudaStream_t)stream) != cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 1;
+  ctx->shard_expanded = 1;
+  ctx->shard_vocab = vocab_count;
+  return C2T_OK;
+}
+
+int c2t_export_row_records(c2t_ctx *ctx, int level, int32_t vocab_begin, c2t_row_record *records_dev,
+                           void *stream) {
+  if (!ctx || !records_dev) return C2T_EINVAL;
+  if (!ctx->shard_expanded || level != ctx->next_level) return C2T_EORDER;
+  if (vocab_begin < 0 || (int64_t)vocab_begin + ctx->shard_vocab > ctx->cfg.vocab) return C2T_EINVAL;
+  if (launch_export_rows(ctx->t, level, ctx->shard_vocab, vocab_begin, records_dev, (cudaStream_t)stream) !=
+      cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 1;
+  ctx->shard_expanded = 0;
+  return C2T_OK;
+}
+
+int c2t_prune_gathered(c2t_ctx *ctx, int level, const c2t_row_record *records_dev, int32_t n_shards,
+                       const c2t_frontier *out, void *stream) {
+  if (!ctx || !records_dev) return C2T_EINVAL;
+  if (n_shards < 1) return C2T_EINVAL;
+  if (n_shards > C2T_MAX_SHARDS) return C2T_ERANGE;
+  if (!ctx->started || ctx->finalized || ctx->expanded || ctx->shard_expanded || level != ctx->next_level ||
+      level >= ctx->cfg.max_depth)
+    return C2T_EORDER;
+  if (launch_prune_level(ctx->t, level, out, records_dev, n_shards, (cudaStream_t)stream) != cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 1;
   ctx->next_level = level + 1;
   return C2T_OK;
 }

@@ -162,7 +162,11 @@ cudaError_t launch_topm_entropy(const void *logits, int64_t seq_stride, int64_t 
                                 cudaStream_t s);
 cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
                               cudaStream_t s);
-cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s);
+// records == nullptr: rows merged from this context's own expand pass; else from n_shards gathered records per row
+cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, const c2t_row_record *records,
+                               int n_shards, cudaStream_t s);
+cudaError_t launch_export_rows(const TreeState &t, int level, int vocab_count, int vocab_begin, c2t_row_record *out,
+                               cudaStream_t s);
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s);
 cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s);
 cudaError_t launch_dense_mask(const TreeState &t, void *out, int out_dtype, int64_t kv_len, cudaStream_t s);

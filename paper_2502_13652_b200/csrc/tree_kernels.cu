@@ -78,7 +78,218 @@ __device__ double classify(const TreeState &t, const float *s_w, double P, doubl
   return 1.0 / (1.0 + exp(-z));
 }
 
-__global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, int level, c2t_frontier out) {
+// What one warp makes of the partial records of one active row of the last expand pass.
+struct RowMerge {
+  double M, S, T;              // row maximum; sums over every other element of e^(x - M) and e^(x - M)(x - M)
+  unsigned long long top;      // the row's best key (0: none)
+  int n_valid;                 // candidates written (at most K)
+};
+
+// One warp merges the partial records of active row `a` (all lanes return the same values).  The K
+// best (logit, token) pairs go to out_x / out_tok (shared or global memory, best first, padded with
+// -inf / -1), token ids offset by tok_base; vloc is the length of the rows the pass read (tokens at
+// or past it pad a ragged last vector).  sk: the warp's staging area of kStageKeys keys.
+__device__ RowMerge merge_row_partials(const TreeState &t, const PassInfo &info, int a, int K, int vloc,
+                                       unsigned long long *sk, float *out_x, int *out_tok, int tok_base) {
+  const int lane = threadIdx.x & 31;
+  // the workers that hold a piece of this row: the rows, each behind info.pad virtual vectors, were cut every info.span
+  const long long first_vec = (long long)a * (info.vec_per_row + info.pad) + info.pad;
+  const int c_first = (int)(first_vec / info.span);
+  const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
+  int n_splits = c_last - c_first + 1;
+  if (n_splits > t.max_splits) n_splits = t.max_splits;
+  const size_t slot0 = (size_t)a * t.max_splits;
+  const int n_keys = n_splits * K;
+
+  // rows with few partials (the usual case): every load is issued before the first use
+  const bool staged = n_splits <= 32 && n_keys <= kStageKeys && kHeldPerSlot == 1;
+  unsigned long long my_held = 0ull;
+  float4 my_stats = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (staged) {
+    if (lane < n_splits) {
+      my_held = t.part_held[slot0 + lane];
+      my_stats = t.part_stats[slot0 + lane];
+    }
+    for (int i = lane; i < n_keys; i += 32) sk[i] = t.part_keys[slot0 * K + i];
+  }
+
+  // the row maximum is the largest key held out of any partial's sums
+  const int n_held = n_splits * kHeldPerSlot;
+  unsigned long long top = my_held;
+  if (!staged) {
+    for (int i = lane; i < n_held; i += 32) {
+      unsigned long long k0 = t.part_held[slot0 * kHeldPerSlot + i];
+      top = k0 > top ? k0 : top;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned long long other = __shfl_xor_sync(kFull, top, o);
+    top = other > top ? other : top;
+  }
+  const double M = (double)key_value(top);
+
+  // fp32 sums of every split: S = sum 2^t, U = sum 2^t t with t = x log2(e) + c, brought to
+  // natural units relative to M:  x - M = t ln2 + g,  g = -c ln2 - M
+  double S = 0.0, T = 0.0;
+  for (int i = lane; i < n_splits; i += 32) {
+    const float4 st = staged ? my_stats : t.part_stats[slot0 + i];
+    const double Ss = (double)st.y, Us = (double)st.z;
+    if (Ss != 0.0 || Us != 0.0) {               // (NaN passes this test and poisons the sums)
+      const double kLn2 = 0.69314718055994530942;
+      const double g = -(double)st.x * kLn2 - M;
+      const double f = exp(g);
+      S += Ss * f;
+      T += f * (kLn2 * Us + g * Ss);
+    }
+  }
+  // held-out elements are not in those sums: add them exactly, all but the row maximum itself
+  for (int i = lane; i < n_held; i += 32) {
+    const unsigned long long key = staged ? my_held : t.part_held[slot0 * kHeldPerSlot + i];
+    if (key == 0ull || key == top) continue;
+    const float x = key_value(key);
+    if (x > kNegInfAsFinite) {
+      double d = (double)x - M;
+      double e = exp(d);
+      S += e;
+      T += e * d;
+    }
+  }
+  // the K best keys over all splits become the candidates
+  S = warp_sum(S);
+  T = warp_sum(T);
+  int n_valid = 0;
+  if (staged) {
+    // every split's list is sorted and now in shared memory, one list per lane: take the
+    // largest head K times (a key of a token past the vocabulary ends its list: it pads a
+    // ragged last vector and sorts behind every real element)
+    __syncwarp();
+    int pos = 0;
+    for (; n_valid < K; ++n_valid) {
+      unsigned long long h = (lane < n_splits && pos < K) ? sk[lane * K + pos] : 0ull;
+      if (h != 0ull && key_token(h) >= vloc) h = 0ull;
+      const uint32_t hi = (uint32_t)(h >> 32), mx_hi = __reduce_max_sync(kFull, hi);
+      const uint32_t mx_lo = __reduce_max_sync(kFull, hi == mx_hi ? (uint32_t)h : 0u);
+      const unsigned long long mx = ((unsigned long long)mx_hi << 32) | mx_lo;
+      if (mx == 0ull) break;
+      if (lane == 0) { out_x[n_valid] = key_value(mx); out_tok[n_valid] = key_token(mx) + tok_base; }
+      if (h == mx) ++pos;
+    }
+    __syncwarp();
+  } else {
+    for (int i = lane; i < n_keys; i += 32) {
+      const unsigned long long key = t.part_keys[slot0 * K + i];
+      if (key == 0ull) continue;
+      const int tok = key_token(key);
+      if (tok >= vloc) continue;                    // padding of a ragged last vector
+      int rank = 0;
+      for (int r = 0; r < n_keys; ++r) {
+        unsigned long long other = t.part_keys[slot0 * K + r];
+        rank += (other > key) && (key_token(other) < vloc);
+      }
+      if (rank < K) { out_x[rank] = key_value(key); out_tok[rank] = tok + tok_base; }
+    }
+    for (int i = lane; i < n_keys; i += 32) {
+      unsigned long long key = t.part_keys[slot0 * K + i];
+      n_valid += (key != 0ull && key_token(key) < vloc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n_valid += __shfl_xor_sync(kFull, n_valid, o);
+    if (n_valid > K) n_valid = K;
+  }
+  // candidates that do not exist (fewer than K tokens in the vocabulary)
+  for (int r = n_valid + lane; r < K; r += 32) { out_x[r] = -INFINITY; out_tok[r] = -1; }
+  RowMerge m;
+  m.M = M; m.S = S; m.T = T; m.top = top; m.n_valid = n_valid;
+  return m;
+}
+
+// status bits of a row from its best key and its sums
+__device__ __forceinline__ uint32_t row_fault_bits(unsigned long long top, double S, double T) {
+  const float top_x = key_value(top);
+  if (top == 0ull || top_x <= kNegInfAsFinite) return C2T_ST_ALL_NEGINF;
+  if (top_x == INFINITY) return C2T_ST_POSINF_LOGIT;
+  if (S != S || T != T || isinf(S)) return C2T_ST_NAN_LOGIT;
+  return 0u;
+}
+
+// One warp merges the gathered records of row (b, j): lane s holds shard s's record.  Writes the K
+// best candidates to out_x / out_tok and returns the merged maximum and sums; *fault_out collects the
+// shards' status bits ("all -inf" only if every shard says so).
+__device__ RowMerge merge_row_records(const TreeState &t, const c2t_row_record *records, int n_shards, int b, int j,
+                                      int K, float *out_x, int *out_tok, uint32_t *fault_out) {
+  const int lane = threadIdx.x & 31;
+  const c2t_row_record *rec = records + ((size_t)lane * t.B + b) * t.F + j;
+  double Mg = 0.0, Sg = 0.0, Tg = 0.0;
+  int ng = 0;
+  uint32_t fg = 0u;
+  bool live = false;
+  if (lane < n_shards) {
+    Mg = rec->M; Sg = rec->S; Tg = rec->T; ng = rec->n; fg = rec->fault;
+    ng = ng < 0 ? 0 : (ng > K ? K : ng);
+    live = !(fg & C2T_ST_ALL_NEGINF);
+  }
+  const uint32_t fault = __reduce_or_sync(kFull, fg & ~(uint32_t)C2T_ST_ALL_NEGINF);
+  // the row maximum is the best of the shards' maxima; equal values go to the lower shard, whose token ids are lower
+  unsigned long long top = live ? (((unsigned long long)f32_orderable(__float_as_uint((float)Mg)) << 32) |
+                                   (0xFFFFFFFFu - (uint32_t)lane)) : 0ull;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned long long other = __shfl_xor_sync(kFull, top, o);
+    top = other > top ? other : top;
+  }
+  const int winner = (int)(0xFFFFFFFFu - (uint32_t)top);
+  const double M = (double)key_value(top);
+  double S = 0.0, T = 0.0;
+  if (live) {
+    const double d = Mg - M, f = exp(d);          // this shard's sums are relative to its own maximum
+    S = f * Sg;
+    T = f * (Tg + d * Sg);
+    if (lane != winner) { S += f; T += f * d; }   // its maximum is an ordinary element of the row
+  }
+  S = warp_sum(S);
+  T = warp_sum(T);
+  int n_valid = 0, pos = 0;
+  for (; n_valid < K; ++n_valid) {                // the shards' lists are sorted: take the largest head K times
+    const unsigned long long h = (live && pos < ng) ? make_key(rec->x[pos], (uint32_t)rec->tok[pos]) : 0ull;
+    const uint32_t hi = (uint32_t)(h >> 32), mx_hi = __reduce_max_sync(kFull, hi);
+    const uint32_t mx_lo = __reduce_max_sync(kFull, hi == mx_hi ? (uint32_t)h : 0u);
+    const unsigned long long mx = ((unsigned long long)mx_hi << 32) | mx_lo;
+    if (mx == 0ull) break;
+    if (lane == 0) { out_x[n_valid] = key_value(mx); out_tok[n_valid] = key_token(mx); }
+    if (h == mx) ++pos;
+  }
+  for (int r = n_valid + lane; r < K; r += 32) { out_x[r] = -INFINITY; out_tok[r] = -1; }
+  *fault_out = fault;
+  RowMerge m;
+  m.M = M; m.S = S; m.T = T; m.top = top; m.n_valid = n_valid;
+  return m;
+}
+
+// The record of every active row of the last (sharded) expand pass, for c2t_export_row_records.
+__global__ void __launch_bounds__(kTreeThreads) export_rows_kernel(TreeState t, int level, int vloc, int tok_base,
+                                                                   c2t_row_record *out) {
+  __shared__ unsigned long long s_keys[kTreeWarps][kStageKeys];
+  chain_enter();
+  const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int n = t.frontier_n[level & 1][b];
+  const int row_off = t.row_off_draft[b];
+  const PassInfo info = *t.info_draft;
+  n = n < 0 ? 0 : (n > t.F ? t.F : n);
+  for (int j = warp; j < n; j += kTreeWarps) {
+    c2t_row_record *r = out + (size_t)b * t.F + j;
+    const RowMerge m = merge_row_partials(t, info, row_off + j, t.K, vloc, s_keys[warp], r->x, r->tok, tok_base);
+    if (lane == 0) {
+      r->M = m.M; r->S = m.S; r->T = m.T;
+      r->n = m.n_valid;
+      r->fault = row_fault_bits(m.top, m.S, m.T);
+    }
+  }
+}
+
+// records == nullptr: the rows come from this context's own expand pass; else from gathered records of n_shards shards
+__global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, int level, c2t_frontier out,
+                                                                   const c2t_row_record *records, int n_shards) {
   __shared__ float s_w[5 * C2T_MAX_HIDDEN + 4];
   __shared__ double s_rowM[C2T_MAX_FRONTIER], s_rowL[C2T_MAX_FRONTIER], s_rowH[C2T_MAX_FRONTIER];
   __shared__ int s_rowfault[C2T_MAX_FRONTIER];
@@ -126,130 +337,20 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
 
   // ---- phase 1: one warp per row merges that row's partial records
   for (int j = warp; j < n; j += kTreeWarps) {
-    const int a = row_off + j;
-    // the workers that hold a piece of this row: the rows, each behind info.pad virtual vectors, were cut every info.span
-    const long long first_vec = (long long)a * (info.vec_per_row + info.pad) + info.pad;
-    const int c_first = (int)(first_vec / info.span);
-    const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
-    int n_splits = c_last - c_first + 1;
-    if (n_splits > t.max_splits) n_splits = t.max_splits;
-    const size_t slot0 = (size_t)a * t.max_splits;
-    const int n_keys = n_splits * K;
-
-    // rows with few partials (the usual case): every load is issued before the first use
-    const bool staged = n_splits <= 32 && n_keys <= kStageKeys && kHeldPerSlot == 1;
-    unsigned long long my_held = 0ull;
-    float4 my_stats = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (staged) {
-      if (lane < n_splits) {
-        my_held = t.part_held[slot0 + lane];
-        my_stats = t.part_stats[slot0 + lane];
-      }
-      unsigned long long *sk = s_keys[warp];
-      for (int i = lane; i < n_keys; i += 32) sk[i] = t.part_keys[slot0 * K + i];
-    }
-
-    // the row maximum is the largest key held out of any partial's sums
-    const int n_held = n_splits * kHeldPerSlot;
-    unsigned long long top = my_held;
-    if (!staged) {
-      for (int i = lane; i < n_held; i += 32) {
-        unsigned long long k0 = t.part_held[slot0 * kHeldPerSlot + i];
-        top = k0 > top ? k0 : top;
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      unsigned long long other = __shfl_xor_sync(kFull, top, o);
-      top = other > top ? other : top;
-    }
-    const double M = (double)key_value(top);
-
-    // fp32 sums of every split: S = sum 2^t, U = sum 2^t t with t = x log2(e) + c, brought to
-    // natural units relative to M:  x - M = t ln2 + g,  g = -c ln2 - M
-    double S = 0.0, T = 0.0;
-    for (int i = lane; i < n_splits; i += 32) {
-      const float4 st = staged ? my_stats : t.part_stats[slot0 + i];
-      const double Ss = (double)st.y, Us = (double)st.z;
-      if (Ss != 0.0 || Us != 0.0) {               // (NaN passes this test and poisons the sums)
-        const double kLn2 = 0.69314718055994530942;
-        const double g = -(double)st.x * kLn2 - M;
-        const double f = exp(g);
-        S += Ss * f;
-        T += f * (kLn2 * Us + g * Ss);
-      }
-    }
-    // held-out elements are not in those sums: add them exactly, all but the row maximum itself
-    for (int i = lane; i < n_held; i += 32) {
-      const unsigned long long key = staged ? my_held : t.part_held[slot0 * kHeldPerSlot + i];
-      if (key == 0ull || key == top) continue;
-      const float x = key_value(key);
-      if (x > kNegInfAsFinite) {
-        double d = (double)x - M;
-        double e = exp(d);
-        S += e;
-        T += e * d;
-      }
-    }
-    // the K best keys over all splits become the candidates
-    S = warp_sum(S);
-    T = warp_sum(T);
-    int n_valid = 0;
-    if (staged) {
-      // every split's list is sorted and now in shared memory, one list per lane: take the
-      // largest head K times (a key of a token past the vocabulary ends its list: it pads a
-      // ragged last vector and sorts behind every real element)
-      const unsigned long long *sk = s_keys[warp];
-      __syncwarp();
-      int pos = 0;
-      for (; n_valid < K; ++n_valid) {
-        unsigned long long h = (lane < n_splits && pos < K) ? sk[lane * K + pos] : 0ull;
-        if (h != 0ull && key_token(h) >= t.V) h = 0ull;
-        const uint32_t hi = (uint32_t)(h >> 32), mx_hi = __reduce_max_sync(kFull, hi);
-        const uint32_t mx_lo = __reduce_max_sync(kFull, hi == mx_hi ? (uint32_t)h : 0u);
-        const unsigned long long mx = ((unsigned long long)mx_hi << 32) | mx_lo;
-        if (mx == 0ull) break;
-        if (lane == 0) { s_x[j * K + n_valid] = key_value(mx); s_tok[j * K + n_valid] = key_token(mx); }
-        if (h == mx) ++pos;
-      }
-      __syncwarp();
-    } else {
-      for (int i = lane; i < n_keys; i += 32) {
-        const unsigned long long key = t.part_keys[slot0 * K + i];
-        if (key == 0ull) continue;
-        const int tok = key_token(key);
-        if (tok >= t.V) continue;                   // padding of a ragged last vector
-        int rank = 0;
-        for (int r = 0; r < n_keys; ++r) {
-          unsigned long long other = t.part_keys[slot0 * K + r];
-          rank += (other > key) && (key_token(other) < t.V);
-        }
-        if (rank < K) { s_x[j * K + rank] = key_value(key); s_tok[j * K + rank] = tok; }
-      }
-      for (int i = lane; i < n_keys; i += 32) {
-        unsigned long long key = t.part_keys[slot0 * K + i];
-        n_valid += (key != 0ull && key_token(key) < t.V);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) n_valid += __shfl_xor_sync(kFull, n_valid, o);
-    }
-    // candidates that do not exist (fewer than K tokens in the vocabulary)
-    for (int r = (n_valid < K ? n_valid : K) + lane; r < K; r += 32) { s_x[j * K + r] = -INFINITY; s_tok[j * K + r] = -1; }
-
+    uint32_t shard_faults = 0u;
+    const RowMerge m = records
+        ? merge_row_records(t, records, n_shards, b, j, K, &s_x[j * K], &s_tok[j * K], &shard_faults)
+        : merge_row_partials(t, info, row_off + j, K, t.V, s_keys[warp], &s_x[j * K], &s_tok[j * K], 0);
     if (lane == 0) {
-      uint32_t fault = 0;
-      const float top_x = key_value(top);
-      if (top == 0ull || top_x <= kNegInfAsFinite) fault |= C2T_ST_ALL_NEGINF;
-      else if (top_x == INFINITY) fault |= C2T_ST_POSINF_LOGIT;
-      else if (S != S || T != T || isinf(S)) fault |= C2T_ST_NAN_LOGIT;
-      const double L = log1p(S);                  // ln sum_v e^(x_v - M); the maximum contributes the 1
-      s_rowM[j] = M;
+      const uint32_t fault = shard_faults ? shard_faults : row_fault_bits(m.top, m.S, m.T);
+      const double L = log1p(m.S);                // ln sum_v e^(x_v - M); the maximum contributes the 1
+      s_rowM[j] = m.M;
       s_rowL[j] = L;
       if (t.entropy_top_m > 0 && t.entropy_top_m < t.V) {
         const double2 sm = t.topm[(size_t)b * F + j];               // Eq. 3: only the M most probable tokens,
-        s_rowH[j] = (L * sm.x - sm.y) / (1.0 + S);                 // probabilities of the full softmax
+        s_rowH[j] = (L * sm.x - sm.y) / (1.0 + m.S);               // probabilities of the full softmax
       } else {
-        s_rowH[j] = L - T / (1.0 + S);            // Eq. 2 with natural log
+        s_rowH[j] = L - m.T / (1.0 + m.S);        // Eq. 2 with natural log
       }
       s_rowfault[j] = (int)fault;
       if (fault) atomicOr(&t.status[b], fault);
@@ -687,10 +788,16 @@ cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const
   return launch_chained(begin_step_kernel, dim3((t.B + 127) / 128), dim3(128), 0, s, t, root_tok, prefix_len);
 }
 
-cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, cudaStream_t s) {
+cudaError_t launch_export_rows(const TreeState &t, int level, int vocab_count, int vocab_begin, c2t_row_record *out,
+                               cudaStream_t s) {
+  return launch_chained(export_rows_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, level, vocab_count, vocab_begin, out);
+}
+
+cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier *out, const c2t_row_record *records,
+                               int n_shards, cudaStream_t s) {
   c2t_frontier o = {nullptr, nullptr, nullptr, nullptr};
   if (out) o = *out;
-  return launch_chained(prune_level_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, level, o);
+  return launch_chained(prune_level_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, level, o, records, n_shards);
 }
 
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s) {

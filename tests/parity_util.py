@@ -108,8 +108,13 @@ def _near_tie_budget(tree, N) -> bool:
 
 
 def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, ctx=None,
-                    draft_dev=None, target_dev=None, check_levels=True) -> Report:
+                    draft_dev=None, target_dev=None, check_levels=True, shards=None) -> Report:
     """Runs one decode step on the GPU (level by level) and on the oracle; asserts parity.
+
+    shards: token ranges [(begin, end), ...] covering the vocabulary in ascending order.  Every level
+    is then built the vocabulary-parallel way (one sharded pass and one record export per range, run
+    one after the other on this GPU, then the prune from the gathered records); the oracle still
+    works on whole rows.
 
     draft_cpu: list of D tensors [B,F,V] on CPU (or None when `seqs` rows are pulled from
     draft_dev); seqs: sequences the oracle checks (default all)."""
@@ -147,9 +152,16 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
 
     root_d = root.to(dev); prefix_d = prefix.to(dev)
     ctx.c2t_begin_step(root_d, prefix_d)
+    records = ctx.new_row_records(len(shards)) if shards else None
     for l in range(D):
-        ctx.c2t_expand_level(l, draft_dev[l])
-        ctx.c2t_prune(l)
+        if shards:
+            for g, (v0, v1) in enumerate(shards):
+                ctx.c2t_expand_level_shard(l, draft_dev[l][:, :, v0:v1])
+                ctx.c2t_export_row_records(l, v0, records[g])
+            ctx.c2t_prune_gathered(l, records)
+        else:
+            ctx.c2t_expand_level(l, draft_dev[l])
+            ctx.c2t_prune(l)
         if not check_levels:
             continue
         view = ctx.c2t_get_view()

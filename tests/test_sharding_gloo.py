@@ -73,3 +73,103 @@ def test_two_ranks_shard_sequences_and_time_by_the_slowest():
     b = c2t_inputs.draft_logits(2, 3, 512, 0, 1, torch.float32, seq_base=2)
     assert torch.equal(a, b)
     assert os.path.isdir(oracle_dir)
+
+
+# ---------------------------------------------------------------- vocabulary-parallel exchange
+
+RECORD = np.dtype([("M", "<f8"), ("S", "<f8"), ("T", "<f8"), ("n", "<i4"), ("fault", "<u4"),
+                   ("tok", "<i4", (32,)), ("x", "<f4", (32,))])
+
+
+def _range_records(logits: torch.Tensor, v0: int, v1: int, K: int) -> np.ndarray:
+    """What a rank exports for its token range [v0, v1) of rows [B, F, V] (plain numpy, fp64)."""
+    x = logits[:, :, v0:v1].double().numpy()
+    B, F, _ = x.shape
+    rec = np.zeros((B, F), dtype=RECORD)
+    for b in range(B):
+        for j in range(F):
+            row = x[b, j]
+            order = np.lexsort((np.arange(row.size), -row))          # logit descending, token id ascending
+            m = row[order[0]]
+            rest = np.delete(row, order[0])
+            rec[b, j]["M"] = m
+            rec[b, j]["S"] = np.exp(rest - m).sum()
+            rec[b, j]["T"] = (np.exp(rest - m) * (rest - m)).sum()
+            k = min(K, row.size)
+            rec[b, j]["n"] = k
+            rec[b, j]["tok"][:k] = order[:k] + v0
+            rec[b, j]["x"][:k] = row[order[:k]]
+    return rec
+
+
+def _vp_worker(rank: int, world: int, port: int, out):
+    sys.path.insert(0, ROOT)
+    import c2t_inputs
+    from paper_2502_13652_b200 import vocab_parallel as vp
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    B, F, V, K = 2, 3, 1000, 5
+    logits = c2t_inputs.draft_logits(B, F, V, 0, 1, torch.float32)    # every rank can draw the whole rows here
+    v0, v1 = vp.shard_ranges(V, world, 4)[rank]
+    local = torch.from_numpy(_range_records(logits, v0, v1, K).view(np.uint8).reshape(B, F, RECORD.itemsize))
+    gathered = vp.gather_row_records(local)                           # the path's only collective
+    if rank == 0:
+        out.put(gathered.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_exchange_row_records_in_token_order():
+    sys.path.insert(0, ROOT)
+    import c2t_inputs
+    from paper_2502_13652_b200 import binding
+    from paper_2502_13652_b200 import vocab_parallel as vp
+    assert RECORD.itemsize == binding.ROW_RECORD_BYTES == 288
+    for V, world, eb in ((1000, 2, 4), (128256, 8, 2), (37, 3, 2), (32000, 7, 4)):
+        r = vp.shard_ranges(V, world, eb)
+        assert r[0][0] == 0 and r[-1][1] == V and all(a[1] == b[0] for a, b in zip(r, r[1:]))
+        assert all((v0 * eb) % 16 == 0 and v1 > v0 for v0, v1 in r)
+    with np.testing.assert_raises(ValueError):
+        vp.shard_ranges(16, 8, 2)
+
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_vp_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    B, F, V, K = 2, 3, 1000, 5
+    logits = c2t_inputs.draft_logits(B, F, V, 0, 1, torch.float32)
+    ranges = vp.shard_ranges(V, 2, 4)
+    assert got.shape == (2, B, F, 288)
+    rec = got.reshape(2, B, F, 288).view(RECORD).reshape(2, B, F)
+    for g, (v0, v1) in enumerate(ranges):                             # shard-major, in rank = token order
+        want = _range_records(logits, v0, v1, K)
+        for name in RECORD.names:
+            assert np.array_equal(rec[g][name], want[name]), (g, name)
+    # merging the two records of a row the way the header states gives the whole row's softmax normaliser,
+    # entropy and top-K (scipy on the whole row)
+    from scipy.special import logsumexp
+    from scipy.stats import entropy
+    for b in range(B):
+        for j in range(F):
+            row = logits[b, j].double().numpy()
+            M = max(rec[g, b, j]["M"] for g in range(2))
+            w = min(g for g in range(2) if rec[g, b, j]["M"] == M)
+            S = T = 0.0
+            for g in range(2):
+                d = rec[g, b, j]["M"] - M
+                S += np.exp(d) * rec[g, b, j]["S"] + (np.exp(d) if g != w else 0.0)
+                T += np.exp(d) * (rec[g, b, j]["T"] + d * rec[g, b, j]["S"]) + (np.exp(d) * d if g != w else 0.0)
+            assert abs((M + np.log1p(S)) - logsumexp(row)) < 1e-12 * abs(logsumexp(row)) + 1e-12
+            p = np.exp(row - logsumexp(row))
+            assert abs((np.log1p(S) - T / (1.0 + S)) - entropy(p)) < 1e-10
+            heads = sorted(((-rec[g, b, j]["x"][i], rec[g, b, j]["tok"][i]) for g in range(2) for i in range(K)))[:K]
+            order = np.lexsort((np.arange(V), -row))[:K]
+            assert [t for _, t in heads] == list(order)
