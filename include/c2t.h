@@ -273,6 +273,22 @@ int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride,
                int64_t row_stride, const c2t_accept_out *out, void *stream);
 
 /*
+ * Greedy acceptance with the target logits sharded over the vocabulary (Sec. 5 Metrics; see
+ * "Vocabulary-parallel levels" above).  c2t_argmax_shard reads this rank's token range
+ * [vocab_begin, vocab_begin + vocab_count) of every final node's row ([B, Nw, vocab_count], strides and
+ * alignment as in c2t_accept with row_stride >= vocab_count) and writes one 64-bit key per node to
+ * keys_dev[b * Nw + i]: the range's largest logit in an order-preserving image in the high word,
+ * 0xFFFFFFFF - (global token id) in the low word, 0 for i >= n_nodes(b).  The caller all-gathers the
+ * keys of all ranges ([n_shards, B, Nw]); c2t_accept_gathered takes the largest key per node (equal
+ * logits: the lower token id), then walks as c2t_accept does; outputs and node_argmax as there.
+ * Both must follow c2t_prune(C2T_FINAL).
+ */
+int c2t_argmax_shard(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, int64_t row_stride,
+                     int32_t vocab_count, int32_t vocab_begin, uint64_t *keys_dev, void *stream);
+int c2t_accept_gathered(c2t_ctx *ctx, const uint64_t *keys_dev, int32_t n_shards, const c2t_accept_out *out,
+                        void *stream);
+
+/*
  * The same greedy acceptance (Sec. 5 Metrics), reading only the target rows the walk visits:
  * the arg-max of the root's row, then of the accepted child's row, and so on, one row per
  * sequence and depth, accept_len + 1 rows per sequence instead of all n_nodes.  Arguments,

@@ -12,4 +12,4 @@ from .binding import (  # noqa: F401
     ST_NAN_LOGIT, ST_POSINF_LOGIT, ST_ALL_NEGINF, ST_TREE_OVERFLOW,
 )
 from .weights import save_classifier, load_classifier  # noqa: F401,E402
-from .vocab_parallel import shard_ranges, gather_row_records, vocab_parallel_level  # noqa: F401,E402
+from .vocab_parallel import shard_ranges, gather_row_records, vocab_parallel_level, vocab_parallel_accept  # noqa: F401,E402

@@ -121,6 +121,11 @@ def lib() -> C.CDLL:
         L.c2t_export_row_records.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_void_p]
         L.c2t_prune_gathered.restype = C.c_int
         L.c2t_prune_gathered.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int32, P(c2t_frontier), C.c_void_p]
+        L.c2t_argmax_shard.restype = C.c_int
+        L.c2t_argmax_shard.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_void_p,
+                                       C.c_void_p]
+        L.c2t_accept_gathered.restype = C.c_int
+        L.c2t_accept_gathered.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, P(c2t_accept_out), C.c_void_p]
         L.c2t_build_verify.restype = C.c_int
         L.c2t_build_verify.argtypes = [C.c_void_p, P(c2t_verify), C.c_void_p]
         L.c2t_accept.restype = C.c_int
@@ -347,6 +352,23 @@ class Context:
         assert t.shape[0] == self.B and t.shape[2] == self.V and t.stride(2) == 1
         _check(lib().c2t_accept(self._h, t.data_ptr(), t.stride(0), t.stride(1), C.byref(self._accept_c),
                                 _stream(stream)), "c2t_accept")
+
+    def c2t_argmax_shard(self, target_shard: torch.Tensor, vocab_begin: int, keys: torch.Tensor, stream=None) -> None:
+        """target_shard: [B, >=Nw, vocab_count] CUDA tensor of the configured dtype; keys: [B, Nw] int64 CUDA
+        tensor (the 64-bit keys, as raw bits)."""
+        t = target_shard
+        assert t.is_cuda and t.dtype == self.cfg.torch_dtype and t.dim() == 3 and t.shape[0] == self.B
+        assert t.stride(2) == 1
+        assert keys.is_cuda and keys.dtype == torch.int64 and keys.is_contiguous() and keys.numel() == self.B * self.Nw
+        _check(lib().c2t_argmax_shard(self._h, t.data_ptr(), t.stride(0), t.stride(1), t.shape[2], vocab_begin,
+                                      keys.data_ptr(), _stream(stream)), "c2t_argmax_shard")
+
+    def c2t_accept_gathered(self, keys: torch.Tensor, stream=None) -> None:
+        """keys: [n_shards, B, Nw] int64 CUDA tensor of gathered keys."""
+        assert keys.is_cuda and keys.dtype == torch.int64 and keys.is_contiguous() and keys.dim() == 3
+        assert keys.shape[1:] == (self.B, self.Nw)
+        _check(lib().c2t_accept_gathered(self._h, keys.data_ptr(), keys.shape[0], C.byref(self._accept_c),
+                                         _stream(stream)), "c2t_accept_gathered")
 
     def c2t_dense_mask(self, out: torch.Tensor, stream=None) -> None:
         """out: [B, Nw, kv_len] CUDA tensor, float32 or bfloat16, contiguous: the additive tree-attention mask."""

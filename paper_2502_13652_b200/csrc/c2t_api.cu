@@ -373,8 +373,48 @@ int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, 
   p.part_best = t.part_best;
   if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, (cudaStream_t)stream) != cudaSuccess)
     return C2T_ECUDA;
-  if (launch_accept_walk(t, out, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
+  if (launch_accept_walk(t, out, nullptr, 0, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
   ctx->launches += 2;
+  return C2T_OK;
+}
+
+int c2t_argmax_shard(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, int64_t row_stride,
+                     int32_t vocab_count, int32_t vocab_begin, uint64_t *keys_dev, void *stream) {
+  if (!ctx || !target_logits_dev || !keys_dev) return C2T_EINVAL;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (vocab_count < 1 || vocab_begin < 0 || (int64_t)vocab_begin + vocab_count > ctx->cfg.vocab || seq_stride < 0 ||
+      row_stride < vocab_count)
+    return C2T_EINVAL;
+  if (!aligned16(target_logits_dev) || (seq_stride * ctx->elem_bytes) % 16 ||
+      (row_stride * ctx->elem_bytes) % 16)
+    return C2T_EALIGN;
+  const TreeState &t = ctx->t;
+  PassParams p;
+  memset(&p, 0, sizeof p);
+  p.logits = target_logits_dev; p.seq_stride = seq_stride; p.row_stride = row_stride;
+  p.V = vocab_count; p.K = 1; p.B = t.B; p.rows_per_seq_max = t.Nw;
+  p.counts = t.final_n;
+  p.max_splits = t.max_splits_tgt;
+  p.info = t.info_target;
+  p.part_best = t.part_best;
+  if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, (cudaStream_t)stream) != cudaSuccess)
+    return C2T_ECUDA;
+  if (launch_export_best(t, vocab_begin, reinterpret_cast<unsigned long long *>(keys_dev), (cudaStream_t)stream) !=
+      cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 2;
+  return C2T_OK;
+}
+
+int c2t_accept_gathered(c2t_ctx *ctx, const uint64_t *keys_dev, int32_t n_shards, const c2t_accept_out *out,
+                        void *stream) {
+  if (!ctx || !keys_dev || n_shards < 1) return C2T_EINVAL;
+  if (n_shards > C2T_MAX_SHARDS) return C2T_ERANGE;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (launch_accept_walk(ctx->t, out, reinterpret_cast<const unsigned long long *>(keys_dev), n_shards,
+                         (cudaStream_t)stream) != cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 1;
   return C2T_OK;
 }
 

@@ -170,7 +170,10 @@ cudaError_t launch_export_rows(const TreeState &t, int level, int vocab_count, i
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s);
 cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaStream_t s);
 cudaError_t launch_dense_mask(const TreeState &t, void *out, int out_dtype, int64_t kv_len, cudaStream_t s);
-cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s);
+// gathered == nullptr: node arg-maxes from this context's own pass; else the best of n_shards gathered keys per node
+cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, const unsigned long long *gathered,
+                               int n_shards, cudaStream_t s);
+cudaError_t launch_export_best(const TreeState &t, int vocab_begin, unsigned long long *out, cudaStream_t s);
 // one round of the lazy walk: round 0 starts it, round r > 0 consumes the arg-max of round r-1
 cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s);
 

@@ -576,7 +576,56 @@ __global__ void __launch_bounds__(kTreeThreads) build_verify_kernel(TreeState t,
 
 // ---------------------------------------------------------------- accept ----
 
-__global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, c2t_accept_out out) {
+// best key of active row `a` of the last arg-max pass (0: none)
+__device__ __forceinline__ unsigned long long row_best_key(const TreeState &t, const PassInfo &info, int a) {
+  const long long first_vec = (long long)a * info.vec_per_row;
+  const int c_first = (int)(first_vec / info.span);
+  const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
+  int n_splits = c_last - c_first + 1;
+  if (n_splits > t.max_splits_tgt) n_splits = t.max_splits_tgt;
+  unsigned long long best = 0ull;
+  for (int s = 0; s < n_splits; ++s) {
+    unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + s];
+    best = k > best ? k : best;
+  }
+  return best;
+}
+
+// rows of earlier sequences in the arg-max pass over the final trees (all threads of the CTA call this)
+__device__ int target_row_offset(const TreeState &t, int b, int *s_scan, int *s_total) {
+  int part = 0;
+  for (int i = threadIdx.x; i < b; i += kTreeThreads) {
+    int c = t.final_n[i];
+    part += c < 0 ? 0 : (c > t.Nw ? t.Nw : c);
+  }
+  int total;
+  block_exclusive_scan(part, s_scan, &total);
+  if (threadIdx.x == 0) *s_total = total;
+  __syncthreads();
+  return *s_total;
+}
+
+// The best key of every final node's row over one token range, token ids made global, for c2t_argmax_shard.
+__global__ void __launch_bounds__(kTreeThreads) export_best_kernel(TreeState t, int tok_base, unsigned long long *out) {
+  __shared__ int s_scan[kTreeWarps + 1];
+  __shared__ int s_total;
+  chain_enter();
+  const int b = blockIdx.x, n = t.final_n[b], Nw = t.Nw;
+  const PassInfo info = *t.info_target;
+  const int row_off = target_row_offset(t, b, s_scan, &s_total);
+  for (int i = threadIdx.x; i < Nw; i += kTreeThreads) {
+    unsigned long long key = 0ull;
+    if (i < n) {
+      const unsigned long long best = row_best_key(t, info, row_off + i);
+      if (best) key = (best & 0xFFFFFFFF00000000ull) | (0xFFFFFFFFu - (uint32_t)(key_token(best) + tok_base));
+    }
+    out[(size_t)b * Nw + i] = key;
+  }
+}
+
+// gathered == nullptr: the arg-max of this context's own pass; else the best of n_shards gathered keys per node
+__global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, c2t_accept_out out,
+                                                                   const unsigned long long *gathered, int n_shards) {
   __shared__ int s_misc[1];
   chain_enter();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -585,7 +634,7 @@ __global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, 
   const PassInfo info = *t.info_target;
 
   // rows of earlier sequences in the argmax pass
-  {
+  if (!gathered) {
     __shared__ int s_scan[kTreeWarps + 1];
     int part = 0;
     for (int i = tid; i < b; i += kTreeThreads) {
@@ -597,21 +646,19 @@ __global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, 
     if (tid == 0) s_misc[0] = total;
     __syncthreads();
   }
-  const int row_off = s_misc[0];
+  const int row_off = gathered ? 0 : s_misc[0];
   // target argmax per node: best key over the row's partials
   for (int i = tid; i < Nw; i += kTreeThreads) {
     int tok = -1;
     if (i < n) {
-      const int a = row_off + i;
-      const long long first_vec = (long long)a * info.vec_per_row;
-      const int c_first = (int)(first_vec / info.span);
-      const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
-      int n_splits = c_last - c_first + 1;
-      if (n_splits > t.max_splits_tgt) n_splits = t.max_splits_tgt;
       unsigned long long best = 0ull;
-      for (int s = 0; s < n_splits; ++s) {
-        unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + s];
-        best = k > best ? k : best;
+      if (gathered) {                               // equal logits in two shards: the larger key is the lower token id
+        for (int s = 0; s < n_shards; ++s) {
+          const unsigned long long k = gathered[((size_t)s * t.B + b) * Nw + i];
+          best = k > best ? k : best;
+        }
+      } else {
+        best = row_best_key(t, info, row_off + i);
       }
       tok = best ? key_token(best) : -1;
     }
@@ -810,10 +857,15 @@ cudaError_t launch_build_verify(const TreeState &t, const c2t_verify *out, cudaS
   return launch_chained(build_verify_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, o);
 }
 
-cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, cudaStream_t s) {
+cudaError_t launch_export_best(const TreeState &t, int vocab_begin, unsigned long long *out, cudaStream_t s) {
+  return launch_chained(export_best_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, vocab_begin, out);
+}
+
+cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, const unsigned long long *gathered,
+                               int n_shards, cudaStream_t s) {
   c2t_accept_out o = {nullptr, nullptr, nullptr};
   if (out) o = *out;
-  return launch_chained(accept_walk_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, o);
+  return launch_chained(accept_walk_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, o, gathered, n_shards);
 }
 
 }  // namespace c2t

@@ -50,3 +50,12 @@ def vocab_parallel_level(ctx, level: int, shard_logits: torch.Tensor, vocab_begi
     ctx.c2t_export_row_records(level, vocab_begin, local, stream)
     records = gather_row_records(local, group)
     ctx.c2t_prune_gathered(level, records, stream)
+
+
+def vocab_parallel_accept(ctx, target_shard: torch.Tensor, vocab_begin: int,
+                          group: Optional[dist.ProcessGroup] = None, stream=None) -> None:
+    """The acceptance walk with sharded target logits: this rank's best key per final node, one all-gather of
+    8 bytes per node, the walk on every rank."""
+    local = torch.zeros((ctx.B, ctx.Nw), dtype=torch.int64, device=target_shard.device)
+    ctx.c2t_argmax_shard(target_shard, vocab_begin, local, stream)
+    ctx.c2t_accept_gathered(gather_row_records(local, group), stream)

@@ -56,6 +56,36 @@ def gen_inputs(B, V, D, F, Nw, dtype, step=0, scale=4.0, device="cpu", seq_base=
     return draft, target, root, prefix
 
 
+# Rows that stress one property each (ties, -inf, a dominant element, values that keep rising).
+def special_rows(kind, B, F, V, dtype):
+    g = torch.Generator().manual_seed(5)
+    if kind == "uniform":
+        return torch.full((B, F, V), 1.5).to(dtype)
+    if kind == "two_valued":
+        x = torch.where(torch.rand(B, F, V, generator=g) < 0.001, torch.tensor(9.0), torch.tensor(-2.0))
+        return x.to(dtype)
+    if kind == "heavy_ties":
+        return (40 + torch.randn(B, F, V, generator=g) * 0.4).to(torch.bfloat16).to(dtype)
+    if kind == "neg_inf":
+        x = torch.randn(B, F, V, generator=g) * 3
+        x[torch.rand(B, F, V, generator=g) < 0.3] = float("-inf")
+        x[:, :, : V // 2] = float("-inf")         # first half of every row has probability zero
+        return x.to(dtype)
+    if kind == "peaked":
+        x = torch.randn(B, F, V, generator=g)
+        x[:, :, 17] = 30.0                         # entropy ~1e-11: the tail must keep relative accuracy
+        return x.to(dtype)
+    if kind == "rising":
+        # every vector beats everything before it; the noise keeps sums of two log-probs from tying
+        x = torch.arange(V, dtype=torch.float32) * (80.0 / V) + torch.randn(B, F, V, generator=g) * 0.3
+        return x.to(dtype)
+    if kind == "late_jump":
+        x = torch.randn(B, F, V, generator=g) - 500.0
+        x[:, :, V - 100:] += 600.0                 # the last elements dwarf everything seen before
+        return x.to(dtype)
+    raise ValueError(kind)
+
+
 @dataclass
 class Report:
     sequences: int = 0
@@ -217,6 +247,18 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
     ctx.c2t_accept_lazy(target_dev)
     acc_l = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
     amax_l = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+    if shards:
+        # the acceptance with the target rows sharded the same way: one key per node and range, the walk from the
+        # gathered keys; everything it writes must equal the whole-row walk (checked against the oracle below)
+        keys = torch.zeros((len(shards), B, ctx.Nw), dtype=torch.int64, device=dev)
+        for g, (v0, v1) in enumerate(shards):
+            ctx.c2t_argmax_shard(target_dev[:, :, v0:v1], v0, keys[g])
+        ctx.c2t_accept_gathered(keys)
+        acc_s = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+        amax_s = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+        for k in acc_g:
+            assert np.array_equal(acc_s[k], acc_g[k]), f"sharded acceptance: {k} differs from the whole-row walk"
+        assert np.array_equal(amax_s, view["node_argmax"])
     ctx.c2t_accept(target_dev)                      # leave the all-rows results behind for the caller
     for b in seqs:
         tree, L, ft, ver, acc = orc[b]

@@ -10,7 +10,7 @@ import torch
 import c2t_inputs
 import oracle
 import paper_2502_13652_b200 as c2t
-from parity_util import RTOL, gen_inputs, make_configs, run_and_compare
+from parity_util import RTOL, gen_inputs, make_configs, run_and_compare, special_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -150,35 +150,6 @@ def test_zero_weights_every_confidence_ties():
 
 def test_wide_limits_k32_f32_h64():
     case(1, 16384, 3, 32, 32, 100, 0.5, torch.bfloat16, hidden=64, wseed=4)
-
-
-def special_rows(kind, B, F, V, dtype):
-    g = torch.Generator().manual_seed(5)
-    if kind == "uniform":
-        return torch.full((B, F, V), 1.5).to(dtype)
-    if kind == "two_valued":
-        x = torch.where(torch.rand(B, F, V, generator=g) < 0.001, torch.tensor(9.0), torch.tensor(-2.0))
-        return x.to(dtype)
-    if kind == "heavy_ties":
-        return (40 + torch.randn(B, F, V, generator=g) * 0.4).to(torch.bfloat16).to(dtype)
-    if kind == "neg_inf":
-        x = torch.randn(B, F, V, generator=g) * 3
-        x[torch.rand(B, F, V, generator=g) < 0.3] = float("-inf")
-        x[:, :, : V // 2] = float("-inf")         # first half of every row has probability zero
-        return x.to(dtype)
-    if kind == "peaked":
-        x = torch.randn(B, F, V, generator=g)
-        x[:, :, 17] = 30.0                         # entropy ~1e-11: the tail must keep relative accuracy
-        return x.to(dtype)
-    if kind == "rising":
-        # every vector beats everything before it; the noise keeps sums of two log-probs from tying
-        x = torch.arange(V, dtype=torch.float32) * (80.0 / V) + torch.randn(B, F, V, generator=g) * 0.3
-        return x.to(dtype)
-    if kind == "late_jump":
-        x = torch.randn(B, F, V, generator=g) - 500.0
-        x[:, :, V - 100:] += 600.0                 # the last elements dwarf everything seen before
-        return x.to(dtype)
-    raise ValueError(kind)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])

@@ -5,8 +5,7 @@ import pytest
 import torch
 
 import paper_2502_13652_b200 as c2t
-from parity_util import gen_inputs, make_configs, run_and_compare
-from test_gpu_parity import special_rows
+from parity_util import gen_inputs, make_configs, run_and_compare, special_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -104,6 +103,17 @@ def test_sharded_faults_and_call_order():
     ctx.c2t_prune_gathered(0, rec)
     bits, per = ctx.c2t_status()
     assert per[0] == 0 and per[1] & c2t.ST_NAN_LOGIT                            # the fault stays with its sequence
+    keys = torch.zeros((2, B, ctx.Nw), dtype=torch.int64, device="cuda")
+    tgt = target.cuda()
+    assert err(ctx.c2t_argmax_shard, tgt[:, :, :2048], 0, keys[0]) == c2t.EORDER   # the tree is not final yet
+    assert err(ctx.c2t_accept_gathered, keys) == c2t.EORDER
+    ctx.c2t_prune(c2t.FINAL)
+    assert err(ctx.c2t_argmax_shard, tgt[:, :, :2048], 2056, keys[0]) == c2t.EINVAL   # range past the vocabulary
+    ctx.c2t_argmax_shard(tgt[:, :, :2048], 0, keys[0])
+    ctx.c2t_argmax_shard(tgt[:, :, 2048:], 2048, keys[1])
+    ctx.c2t_accept_gathered(keys)
+    big_keys = torch.zeros((33, B, ctx.Nw), dtype=torch.int64, device="cuda")
+    assert err(ctx.c2t_accept_gathered, big_keys) == c2t.ERANGE
     ctx.close()
 
     _, mcfg = make_configs(B, V, D, K, F, N, 0.5, torch.float32, M=100)
