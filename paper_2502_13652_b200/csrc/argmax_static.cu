@@ -12,6 +12,8 @@ constexpr int kStaticMaxVocab = C2T_STATIC_MAX_VOCAB;
 // slots per row the arg-max pass can need at the largest vocabulary (fp32: 4 elements per vector)
 constexpr int kStaticMaxSplits = (kStaticMaxVocab / 4 + kMinSpanVectors - 1) / kMinSpanVectors + 1;
 constexpr int kMaxDevices = 64;
+// the arg-max kernel keeps one row offset per "sequence" in shared memory, sized by the batch limit
+static_assert(C2T_STATIC_MAX_ROWS <= C2T_MAX_BATCH, "the static entry point passes its rows as the batch of the pass");
 
 struct StaticScratch {
   PassInfo info;                                              // what the pass derived from the row counts

@@ -26,13 +26,17 @@ def _built():
     assert os.path.exists(c2t.LIB_PATH)
 
 
-def case(B, V, D, K, F, N, beta, dtype, step=0, scale=4.0, **kw):
+def case(B, V, D, K, F, N, beta, dtype, step=0, scale=4.0, allow_diverged=0, allow_kinds=(), **kw):
+    """One decode step of seeded inputs on both sides.  No sequence may differ from the oracle unless the
+    caller names the boundary case and bounds the count (see parity_util)."""
     ocfg, gcfg = make_configs(B, V, D, K, F, N, beta, dtype, **kw)
     Nw = c2t.c2t_final_width(gcfg)
     draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype, step=step, scale=scale)
-    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, allow_diverged=allow_diverged,
+                          allow_kinds=allow_kinds)
     print(f"\n  [{B}x{V} {str(dtype)[6:]} D{D} K{K} F{F} N{N} b{beta}] {rep.line()}")
     assert rep.status_bits == 0
+    assert rep.kept_nodes == rep.oracle_kept_nodes or rep.diverged_sequences
     return rep
 
 
@@ -67,8 +71,7 @@ def test_tiny_hand_enumerated_tree():
 
 
 def test_config1_single_sequence_fp32():
-    rep = case(1, 32000, 6, 10, 10, 60, 0.5, torch.float32)
-    assert rep.diverged_sequences == 0 or rep.near_tie_sequences > 0
+    case(1, 32000, 6, 10, 10, 60, 0.5, torch.float32)
 
 
 def test_config2_batch8_bf16_several_steps():
@@ -121,7 +124,6 @@ def test_chain_mode_stop_rules(rule, thr):
     """K = F = 1 with the three early-stop rules of the chain-mode comparison (Sec. 5): maximum
     probability, joint probability, the classifier.  Chains end at different depths per sequence."""
     rep = case(8, 32000, 10, 1, 1, 0, thr, torch.bfloat16, scale=1.5, classifier=rule, wseed=5)
-    assert rep.diverged_sequences == 0 or rep.near_tie_sequences > 0
     assert len(set(rep.kept_nodes)) >= 2
 
 
@@ -144,8 +146,7 @@ def test_eagle2_complete_tree_1011_nodes():
 
 
 def test_zero_weights_every_confidence_ties():
-    rep = case(2, 8000, 4, 5, 3, 10, 0.5, torch.bfloat16, wstd=0.0)
-    assert rep.diverged_sequences == 0
+    case(2, 8000, 4, 5, 3, 10, 0.5, torch.bfloat16, wstd=0.0)
 
 
 def test_wide_limits_k32_f32_h64():
@@ -161,12 +162,13 @@ def test_special_rows(kind, dtype):
     draft = [special_rows(kind, B, F, V, dtype) for _ in range(D)]
     target = special_rows(kind, B, Nw, V, dtype)
     root = torch.zeros(B, dtype=torch.int32); prefix = torch.full((B,), 9, dtype=torch.int32)
-    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
+    # all-equal rows make the confidences of children of different rows exactly equal in the oracle, which
+    # orders them by candidate index; the CUDA path's fp32 row sums depend on where a row is cut into
+    # segments, so there the order follows the last bits of two sums: the one named departure
+    uniform = dict(allow_diverged=B, allow_kinds=("cross_row_tie",)) if kind == "uniform" else {}
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, **uniform)
     print(f"\n  [{kind} {dtype}] {rep.line()}")
     assert rep.status_bits == 0
-    # all-equal rows tie every candidate exactly in the oracle; the CUDA path's fp32 tail sums depend on
-    # where a row is cut into segments, so there the tie is broken by rounding (a counted near tie)
-    assert rep.diverged_sequences == 0 or (kind == "uniform" and rep.diverged_sequences <= rep.near_tie_sequences)
     if kind == "uniform":
         ctx = c2t.Context(gcfg)
         ctx.c2t_begin_step(root.cuda(), prefix.cuda())
@@ -317,8 +319,7 @@ def test_back_to_back_steps_equal_isolated_steps():
 def test_truncated_entropy_top_m(dtype, V, M):
     """Eq. 3: the entropy feature over the M most probable tokens only (the paper's M = 1000), full
     softmax probabilities; M >= V is the exact entropy again."""
-    rep = case(4, V, 4, 8, 6, 24, 0.5, dtype, M=M)
-    assert rep.diverged_sequences == 0 or rep.near_tie_sequences > 0
+    case(4, V, 4, 8, 6, 24, 0.5, dtype, M=M)
 
 
 @pytest.mark.parametrize("kind", ["heavy_ties", "two_valued", "neg_inf", "uniform"])
@@ -331,9 +332,9 @@ def test_truncated_entropy_on_special_rows(kind):
     draft = [special_rows(kind, B, F, V, dtype) for _ in range(D)]
     target = special_rows(kind, B, Nw, V, dtype)
     root = torch.zeros(B, dtype=torch.int32); prefix = torch.full((B,), 9, dtype=torch.int32)
-    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix)
+    uniform = dict(allow_diverged=B, allow_kinds=("cross_row_tie",)) if kind == "uniform" else {}
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, **uniform)
     assert rep.status_bits == 0
-    assert rep.diverged_sequences == 0 or (kind == "uniform" and rep.diverged_sequences <= rep.near_tie_sequences)
 
 
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])

@@ -14,6 +14,7 @@ import pytest
 import torch
 
 import c2t_inputs
+import oracle
 import paper_2502_13652_b200 as c2t
 from parity_util import gen_inputs, make_configs
 
@@ -51,6 +52,38 @@ def test_static_scratch_argmax_matches_accept_twice_in_a_row(dtype):
         tied = (target.view(B * Nw, V) == target.view(B * Nw, V).max(dim=1, keepdim=True).values).sum(1) > 1
         assert torch.equal(out[~tied], direct[~tied])
     ctx.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_static_scratch_argmax_against_the_oracle_on_tie_heavy_rows(dtype):
+    """Row by row against the oracle's arg-max (largest logit, ties to the lower token id) on rows where
+    the maximum occurs many times, with a row length that is not a whole number of 16-byte vectors, -inf
+    entries and a padded stride.  Two calls in a row with different row counts: the second, shorter call
+    must not see the keys the first one left in the shared scratch."""
+    from paper_2502_13652_b200 import build
+    build.build()
+    oracle.build()
+    V, Vp = 5003, 5024
+    g = torch.Generator().manual_seed(11)
+    for rows in (37, 9):
+        x = (40 + torch.randn(rows, V, generator=g) * 0.4).to(torch.bfloat16)      # spacing 0.25: the maximum repeats
+        x[torch.rand(rows, V, generator=g) < 0.2] = float("-inf")
+        x[rows // 2, :] = float("-inf")                                             # a row without any finite logit
+        x[0, :] = 3.0                                                               # all equal: token 0
+        x = x.to(dtype)
+        assert int((x[1] == x[1].max()).sum()) > 1
+        buf = torch.full((rows, Vp), float("nan"), dtype=dtype, device="cuda")      # the padding must never be read
+        buf[:, :V] = x.cuda()
+        out = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+        c2t.c2t_row_argmax_static(buf[:, :V], out)
+        torch.cuda.synchronize()
+        want = [oracle.row_argmax(x[r]) for r in range(rows)]
+        got = out.tolist()
+        for r in range(rows):
+            if r == rows // 2:
+                continue                                     # all -inf: no arg-max is defined; both sides only stay in range
+            assert got[r] == want[r], (rows, r, got[r], want[r])
+        assert -1 <= got[rows // 2] < V
 
 
 def test_static_scratch_limits_and_arguments():
