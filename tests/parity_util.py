@@ -112,6 +112,7 @@ class Report:
     accept_len: list = field(default_factory=list)         # the CUDA path's accept lengths
     oracle_kept_nodes: list = field(default_factory=list)
     oracle_accept_len: list = field(default_factory=list)
+    oracle_next_token: list = field(default_factory=list)
 
     def line(self) -> str:
         return (f"seq={self.sequences} near_tie={self.near_tie_sequences} diverged={self.diverged_sequences} "
@@ -331,6 +332,7 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
         tree, L, ft, ver, acc = orc[b]
         near[b] = near[b] or _near_tie_budget(tree, ocfg.budget)
         rep.oracle_kept_nodes.append(int(ft.n)); rep.oracle_accept_len.append(int(acc.accept_len))
+        rep.oracle_next_token.append(int(acc.next_token))
         rep.kept_nodes.append(int(ver_g["n_nodes"][b])); rep.accept_len.append(int(acc_g["accept_len"][b]))
         if b in diverged:
             continue
@@ -377,3 +379,61 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
         f"{rep.diverged_sequences} sequence(s) differ from the oracle through boundary cases {rep.where}; "
         f"this case allows {allow_diverged} of kinds {tuple(allow_kinds)}")
     return rep
+
+
+ALL_KINDS = ("near_beta", "near_cap", "near_budget", "cross_row_tie")
+
+
+def run_chain(ocfg, gcfg, n_steps, seqs, scale=4.0, allow_diverged=0, allow_kinds=()):
+    """`n_steps` decode steps in a row: step s + 1 starts from step s's next token and from a prefix
+    that is accept_len + 1 tokens longer (Sec. 2.1: the accepted drafts and the target's own token are
+    committed).  The CUDA path carries that state on the device, from its own outputs; the oracle
+    carries its own.  Before every step the two states of the checked sequences must be equal; every
+    step is compared like a single one.  A step that differs through a boundary case (see the module
+    docstring) is counted, and the oracle's state is set to the CUDA path's from there on."""
+    dtype = gcfg.torch_dtype
+    B, V, D, F = gcfg.batch, gcfg.vocab, gcfg.max_depth, gcfg.frontier_cap
+    ctx = c2t.Context(gcfg)
+    dev = ctx.device
+    Nw = ctx.Nw
+    root = c2t_inputs.root_tokens(B, V, 0).to(dev)
+    prefix = c2t_inputs.prefix_lengths(B).to(dev)
+    o_root = {b: int(root[b]) for b in seqs}
+    o_prefix = {b: int(prefix[b]) for b in seqs}
+    out = Report(sequences=len(seqs))
+    steps_diverged = 0
+    for s in range(n_steps):
+        draft = [c2t_inputs.draft_logits(B, F, V, s, l, dtype, scale, device=dev) for l in range(D)]
+        target = c2t_inputs.target_logits(B, Nw, V, s, dtype, scale, device=dev)
+        rc, pc = root.cpu(), prefix.cpu()
+        for b in seqs:
+            assert int(rc[b]) == o_root[b] and int(pc[b]) == o_prefix[b], f"step {s} seq {b}: the chains' states differ"
+        rep = run_and_compare(ocfg, gcfg, None, None, root, prefix, seqs=seqs, ctx=ctx, draft_dev=draft,
+                              target_dev=target, allow_diverged=len(seqs), allow_kinds=ALL_KINDS)
+        assert rep.status_bits == 0
+        # both chains advance from their own results (device tensors on the CUDA side: no host round trip)
+        new_root = ctx.accepted["next_token"].clone()
+        new_prefix = prefix + ctx.accepted["accept_len"] + 1
+        for i, b in enumerate(seqs):
+            if b in rep.where:
+                steps_diverged += 1
+                out.excused[rep.where[b][1]] = out.excused.get(rep.where[b][1], 0) + 1
+                out.where[(s, b)] = rep.where[b]
+                o_root[b], o_prefix[b] = int(new_root[b]), int(new_prefix[b])
+            else:
+                o_root[b] = rep.oracle_next_token[i]
+                o_prefix[b] += rep.oracle_accept_len[i] + 1
+        root, prefix = new_root, new_prefix
+        out.kept_nodes += rep.kept_nodes; out.accept_len += rep.accept_len
+        out.oracle_kept_nodes += rep.oracle_kept_nodes; out.oracle_accept_len += rep.oracle_accept_len
+        out.max_rel_p = max(out.max_rel_p, rep.max_rel_p); out.max_rel_H = max(out.max_rel_H, rep.max_rel_H)
+        out.max_rel_C = max(out.max_rel_C, rep.max_rel_C)
+        out.near_tie_sequences += rep.near_tie_sequences
+    out.diverged_sequences = steps_diverged
+    out.status_bits = 0
+    out.final_prefix = prefix.cpu()
+    ctx.close()
+    assert steps_diverged <= allow_diverged and set(out.excused) <= set(allow_kinds), (
+        f"{steps_diverged} sequence-step(s) differ from the oracle through boundary cases {out.where}; "
+        f"this chain allows {allow_diverged} of kinds {tuple(allow_kinds)}")
+    return out

@@ -10,7 +10,7 @@ import torch
 import c2t_inputs
 import oracle
 import paper_2502_13652_b200 as c2t
-from parity_util import RTOL, gen_inputs, make_configs, run_and_compare, special_rows
+from parity_util import RTOL, gen_inputs, make_configs, run_and_compare, run_chain, special_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -81,6 +81,38 @@ def test_config2_batch8_bf16_several_steps():
         rep = case(8, 32000, 8, 10, 10, 60, 0.5, torch.bfloat16, step=step)
         nodes += rep.kept_nodes
     assert max(nodes) > 1
+
+
+def test_config2_chained_64_steps():
+    """B=8, V=32000, bf16, D=8, K=F=10, N=60: 64 decode steps in which every step starts from the
+    previous step's next token and grown prefix; two of the eight sequences are checked against the
+    oracle at every step (the oracle needs seconds per sequence and step)."""
+    ocfg, gcfg = make_configs(8, 32000, 8, 10, 10, 60, 0.5, torch.bfloat16)
+    rep = run_chain(ocfg, gcfg, 64, seqs=[1, 6])
+    print(f"\n  [config 2, 64 chained steps] {rep.line()}")
+    assert len(rep.accept_len) == 2 * 64 and rep.accept_len == rep.oracle_accept_len
+    assert rep.kept_nodes == rep.oracle_kept_nodes and max(rep.kept_nodes) > 1
+
+
+# The ablation sweep's corner points at full batch: classifier (identity on the joint probability, i.e.
+# EAGLE-2's expand + rerank, against the FFN), both vocabularies and dtypes, the smallest and largest budget,
+# the deepest tree, the flattest and the most peaked logits.  Sampled sequences, as for the throughput case.
+@pytest.mark.parametrize("V,dtype,classifier,N,scale", [
+    (128256, torch.float32, "identity", 20, 1.0),
+    (128256, torch.bfloat16, "mlp", 80, 8.0),
+    (128256, torch.bfloat16, "identity", 80, 1.0),
+    (32000, torch.float32, "mlp", 20, 8.0),
+    (32000, torch.bfloat16, "identity", 80, 8.0),
+])
+def test_config5_ablation_corners_sampled(V, dtype, classifier, N, scale):
+    B, D, K, F = 32, 10, 10, 10
+    beta = 0.5 if classifier == "mlp" else 0.0
+    ocfg, gcfg = make_configs(B, V, D, K, F, N, beta, dtype, classifier=classifier)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype, scale=scale, device="cuda")
+    rep = run_and_compare(ocfg, gcfg, None, None, root, prefix, seqs=[0, 17], draft_dev=draft, target_dev=target)
+    print(f"\n  [config 5: V={V} {dtype} {classifier} N={N} scale={scale}] {rep.line()}")
+    assert rep.status_bits == 0 and rep.kept_nodes == rep.oracle_kept_nodes
 
 
 @pytest.mark.parametrize("beta", [0.3, 0.5, 0.7])
