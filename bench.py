@@ -15,12 +15,15 @@ scaling, no collective on the data path).  Rank 0 prints one JSON line.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import statistics
 import subprocess
 import sys
 import tempfile
 import time
+from concurrent.futures import ThreadPoolExecutor
 
 import torch
 
@@ -34,13 +37,29 @@ METRIC = "draft-tree levels/sec and µs per decode step; logits HBM GB/s vs ~8 T
 UNIT = "levels/s"
 
 WORKLOAD = dict(B=64, V=128256, D=8, K=10, F=10, N=60, beta=0.5, hidden=16)
+REPEAT_BLOCKS = 6             # further blocks of `steps` steps after the headline block, for median / min / max
 WORKLOAD_NAME = ("B=64 sequences, V=128256, bf16 draft and target logits, depth 8, top-k 10, frontier cap 10, "
                  "budget 60, threshold 0.5, MLP hidden 16")
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one expand_pass_kernel launch at this workload, from the ncu capture summarised in
-# profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  Set to
-# None when the kernel changes until the counters are taken again.
+# profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  The counters
+# belong to the kernel sources whose hash stands beside them: when a source changes the hash no longer matches and
+# the bench reports no traffic figure until the counters (and the hash) are taken again.
 EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.09e6}
+EXPAND_SOURCES = ("expand_pass.cu", "c2t_internal.h", "vocab_common.cuh")
+EXPAND_SOURCES_SHA16 = "d33adf80192b8868"
+
+
+def expand_dram_bytes():
+    """The ncu counters above, or None if the kernel's sources are not the ones they were taken on."""
+    h = hashlib.sha256()
+    try:
+        for name in EXPAND_SOURCES:
+            with open(os.path.join(ROOT, "paper_2502_13652_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+    except OSError:
+        return None
+    return EXPAND_DRAM_BYTES if h.hexdigest()[:16] == EXPAND_SOURCES_SHA16 else None
 
 
 def measured_hbm_peak():
@@ -150,39 +169,75 @@ def oracle_config():
                                w1=w1, b1=b1, w2=w2, b2=b2)
 
 
-def time_oracle(n_seq: int, steps: int, warmup: int):
-    """Seconds per step of the oracle on n_seq sequences (single thread)."""
+def host_cores() -> int:
+    """Cores this process may run on."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def time_oracle(n_seq: int, steps: int, warmup: int, threads: int = 1):
+    """Seconds per step of the oracle, as it stands, on n_seq sequences of the workload: one thread, or `threads`
+    threads that each take whole sequences (the oracle works one sequence at a time and keeps no global state;
+    the calls run outside the interpreter lock).  Returns (seconds per step, logits rows per step)."""
     import oracle
     oracle.build()
-    cfg = oracle_config()
     draft, target, root, prefix = oracle_sample(n_seq)
+    root, prefix = root.numpy(), prefix.numpy()
     for _ in range(warmup):
-        oracle.decode_step(cfg, draft[:1], target[:1], root[:1].numpy(), prefix[:1].numpy())
+        oracle.decode_step(oracle_config(), draft[:1], target[:1], root[:1], prefix[:1])
+
+    def one(b):
+        return oracle.decode_step(oracle_config(), draft[b:b + 1], target[b:b + 1], root[b:b + 1],
+                                  prefix[b:b + 1]).rows_visited
+
     t0 = time.perf_counter()
     rows = 0
     for _ in range(steps):
-        rows += oracle.decode_step(cfg, draft, target, root.numpy(), prefix.numpy()).rows_visited
+        if threads <= 1:
+            rows += oracle.decode_step(oracle_config(), draft, target, root, prefix).rows_visited
+        else:
+            with ThreadPoolExecutor(max_workers=threads) as pool:
+                rows += sum(pool.map(one, range(n_seq)))
     dt = (time.perf_counter() - t0) / steps
     return dt, rows // max(steps, 1)
+
+
+MAX_ORACLE_THREADS = 16      # bounds the sample (one sequence per thread) and the time spent generating it
+
+
+def oracle_baseline(steps: int, warmup: int):
+    """The oracle on this host: threads over sequences on the cores this process may use (at most
+    MAX_ORACLE_THREADS), and on one core.  Returns the `cpu_baseline` object of the JSON line and ms per step."""
+    w = WORKLOAD
+    cores = host_cores()
+    threads = min(cores, MAX_ORACLE_THREADS)
+    n_seq = max(threads, 2)
+    dt, rows = time_oracle(n_seq, steps, warmup, threads)
+    value = n_seq * w["D"] / dt
+    n1 = 2
+    dt1, rows1 = time_oracle(n1, 1, 0, 1)
+    sample = (f"{n_seq} of the workload's {w['B']} sequences per step, one sequence per thread (all {w['D']} levels, "
+              f"rerank, verify inputs, accept walk; {rows} logits rows of {w['V']} bf16 per step), {dt:.1f} s per step")
+    return {"value": value, "unit": UNIT, "cores": threads, "host_cores": cores, "kind": "oracle", "sample": sample,
+            "single_core": {"value": n1 * w["D"] / dt1, "unit": UNIT, "cores": 1,
+                            "sample": f"{n1} sequences, one step ({rows1} logits rows), {dt1:.1f} s"}}, dt * 1e3
 
 
 def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n_seq = 2
-    dt, rows = time_oracle(n_seq, args.steps, min(args.warmup, 1))
-    value = n_seq * WORKLOAD["D"] / dt
-    sample = (f"{n_seq} of the workload's 64 sequences per step (all {WORKLOAD['D']} levels, rerank, verify "
-              f"inputs, accept walk; {rows} logits rows of {WORKLOAD['V']} bf16 per step)")
+    base, ms = oracle_baseline(args.steps, min(args.warmup, 1))
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAME, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "us_per_step": dt * 1e6,
+        "config": {"workload": WORKLOAD_NAME, "sample": base["sample"]},
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "us_per_step": ms * 1e3,
     }
     print(json.dumps(line), flush=True)
 
@@ -222,7 +277,7 @@ def run_cuda(args) -> None:
     prefix = c2t_inputs.prefix_lengths(B, seq_base=seq_base).to(dev)
     default_stream = stream = torch.cuda.current_stream().cuda_stream
 
-    def step(events=None, lazy=False, stream_handle=None):
+    def step(events=None, lazy=False, stream_handle=None, target=target):
         stream = stream_handle if stream_handle is not None else default_stream
         ctx.c2t_begin_step(root, prefix, stream)
         for l in range(D):
@@ -282,11 +337,25 @@ def run_cuda(args) -> None:
     ms_total = e0.elapsed_time(e1)
     expand_ms = sum(evs[s][2 * l].elapsed_time(evs[s][2 * l + 1]) for s in sampled for l in range(D))
     full_ms = [evs[s][2 * l].elapsed_time(evs[s][2 * l + 1]) for s in sampled for l in range(1, D)]
-    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
     ms_total_max = max_over_ranks(ms_total, dist, dev)
     ms_per_step = ms_total_max / args.steps
     value = whole_job_levels_per_second(world, B, D, ms_per_step)
+
+    # ---- the same block of `steps` steps a few more times: median and range beside the headline (which is the
+    # first block, as timed above); the clock samples cover these blocks too
+    block_ms = [ms_per_step]
+    for _ in range(REPEAT_BLOCKS):
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        r0.record()
+        for s in range(args.steps):
+            step()
+        r1.record()
+        barrier()
+        block_ms.append(max_over_ranks(r0.elapsed_time(r1), dist, dev) / args.steps)
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
     # ---- the same steps with the acceptance walk that reads only the rows it visits (reported beside the
     # headline, which keeps the all-rows arg-max of the workload definition)
@@ -301,6 +370,25 @@ def run_cuda(args) -> None:
     barrier()
     lazy_ms_per_step = max_over_ranks(z0.elapsed_time(z1), dist, dev) / args.steps
     assert torch.equal(ctx.accepted["accept_len"].cpu(), accept_len)
+
+    # ---- both acceptance calls on target rows whose arg-maxes follow a path of the final tree (2 to 5 levels
+    # deep, 3.5 on average where the trees allow it): the synthetic target rows alone accept almost nothing, so
+    # the walk never moves and the lazy call reads one row per sequence; with planted paths it reads tau + 1
+    target_planted, planted_depth = plant_accept_paths(ctx, target, V)
+    planted = {}
+    for name, lazy in (("all_rows", False), ("lazy", True)):
+        for _ in range(3):
+            step(lazy=lazy, target=target_planted)
+        barrier()
+        y0, y1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        y0.record()
+        for s in range(args.steps):
+            step(lazy=lazy, target=target_planted)
+        y1.record()
+        barrier()
+        planted[name] = max_over_ranks(y0.elapsed_time(y1), dist, dev) / args.steps
+        assert ctx.accepted["accept_len"].cpu().tolist() == planted_depth
+    del target_planted
 
     # ---- the same step captured once in a CUDA graph and replayed (all-rows accept): what a serving loop
     # without a draft model between the levels would do; reported beside the headline
@@ -356,10 +444,18 @@ def run_cuda(args) -> None:
 
     # ---- the same expand kernel on fp32 logits (twice the bytes per element, the same arithmetic per element):
     # reported beside the bf16 figure to show which side of the kernel the bytes-per-element ratio puts the bound on
-    fp32_level = expand_full_level_fp32(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream)
+    fp32_level = expand_full_level(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream, torch.float32, 4.0)
+    # ... and on flat logits (temperature scale 1), where the kernel's work per element is at its largest
+    scale1_level = expand_full_level(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream, torch.bfloat16, 1.0)
 
     # ---- the single-sequence configuration (latency-bound), timed per decode step; one GPU only
     single_seq = single_sequence_latency(c2t, dev, default_stream) if world == 1 else None
+    configs = None
+    if world == 1:
+        configs = {"config1": config1_single_sequence_fp32(c2t, dev, default_stream),
+                   "config2": config2_chained_steps(c2t, dev, default_stream),
+                   "config3": "single_sequence (below)",
+                   "config5": config5_ablation_sweep(c2t, dev, default_stream)}
 
     # ---- roofline of the dominant kernel (the per-level vocabulary pass)
     peak, peak_kind = measured_hbm_peak()
@@ -376,16 +472,13 @@ def run_cuda(args) -> None:
     # two launch shapes, profiles/expand_pass_kernel_bf16_B64_V128256.txt), scaled by the rows a launch streams
     # and averaged over the step's launches like `achieved`.  None when the counters do not cover the workload.
     traffic = None
-    if (B, V, F) == (64, 128256, 10) and EXPAND_DRAM_BYTES is not None:
-        per_row = [EXPAND_DRAM_BYTES["level0"] / 64.0] + [EXPAND_DRAM_BYTES["full_level"] / 640.0] * (D - 1)
+    dram = expand_dram_bytes()
+    if (B, V, F) == (64, 128256, 10) and dram is not None:
+        per_row = [dram["level0"] / 64.0] + [dram["full_level"] / 640.0] * (D - 1)
         traffic = sum(r * b for r, b in zip(rows_per_level, per_row)) / D
 
     # ---- the oracle on this host, bounded sample
-    n_seq = 8
-    dt_cpu, rows_cpu = time_oracle(n_seq, 1, 1)
-    cpu_value = n_seq * D / dt_cpu
-    sample = (f"{n_seq} of the workload's {B} sequences, one decode step ({rows_cpu} logits rows of {V} bf16), "
-              f"{dt_cpu:.1f} s")
+    cpu_base, _ = oracle_baseline(1, 1)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -397,14 +490,25 @@ def run_cuda(args) -> None:
                    "mean_accept_len": float(accept_len.float().mean()), "status_bits": status,
                    "parallelism": f"dp{world} (independent sequences per rank, no collective)"},
         "us_per_step": ms_per_step * 1e3, "us_per_level": ms_per_step * 1e3 / D,
+        "us_per_step_blocks": {"n": len(block_ms), "steps_per_block": args.steps,
+                               "median": statistics.median(block_ms) * 1e3, "min": min(block_ms) * 1e3,
+                               "max": max(block_ms) * 1e3},
         "graph_replay": None if graph_ms_per_step is None else {
             "us_per_step": graph_ms_per_step * 1e3,
             "value": whole_job_levels_per_second(world, B, D, graph_ms_per_step), "unit": UNIT,
             "note": "the step's 21 launches captured once in a CUDA graph and replayed"},
         "lazy_accept": {"us_per_step": lazy_ms_per_step * 1e3,
                         "value": whole_job_levels_per_second(world, B, D, lazy_ms_per_step), "unit": UNIT,
-                        "note": "c2t_accept_lazy: accept_len+1 target rows per sequence instead of all final nodes"},
+                        "mean_accept_len": float(accept_len.float().mean()),
+                        "note": "c2t_accept_lazy: accept_len+1 target rows per sequence instead of all final nodes",
+                        "planted_paths": {
+                            "mean_accept_len": sum(planted_depth) / len(planted_depth),
+                            "target_rows_read_per_sequence": sum(planted_depth) / len(planted_depth) + 1,
+                            "us_per_step_lazy": planted["lazy"] * 1e3,
+                            "us_per_step_all_rows": planted["all_rows"] * 1e3,
+                            "note": "target arg-maxes planted along a path of each final tree"}},
         "single_sequence": single_seq,
+        "configs": configs,
         "clocks": clocks,
         "e2e": {"value": whole_job_levels_per_second(world, B, D, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -416,26 +520,53 @@ def run_cuda(args) -> None:
                      "avg_launch_us": avg_launch_s * 1e6,
                      "full_level_rows": full_rows, "full_level_gbs": full_level_gbs,
                      "frac_of_8000": achieved / 8000.0,
+                     "us_x_sm_mhz": None if not clocks or not clocks.get("sm_mhz") else
+                     avg_launch_s * 1e6 * clocks["sm_mhz"],
                      "fp32_logits_full_level": None if fp32_level is None else dict(
-                         fp32_level, frac=fp32_level["gbs"] / peak)},
-        "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+                         fp32_level, frac=fp32_level["gbs"] / peak),
+                     "scale1_logits_full_level": None if scale1_level is None else dict(
+                         scale1_level, frac=scale1_level["gbs"] / peak, frac_of_8000=scale1_level["gbs"] / 8000.0)},
+        "cpu_baseline": cpu_base,
     }
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
 
-def expand_full_level_fp32(c2t, dev, weights, root, prefix, stream, reps: int = 20):
-    """Times expand_pass_kernel<fp32> on full levels of the workload with fp32 logits (levels 1-3, three distinct
-    buffers of 328 MB, so every launch reads from DRAM).  Returns None if the frontier does not fill."""
+def plant_accept_paths(ctx, target, V, depths=(2, 3, 4, 5)):
+    """A copy of `target` in which, per sequence, the arg-maxes of the rows along one root-to-leaf path of the final
+    tree (as the context's last step left it) point to the next node of the path, down to a chosen depth, and the
+    row at that depth points to a token none of its children carries.  Returns (tensor, accept length per sequence)."""
+    ver = {k: v.cpu().numpy() for k, v in ctx.verify.items()}
+    out = target.clone()
+    got = []
+    for b in range(ctx.B):
+        n = int(ver["n_nodes"][b])
+        rows = ver["retrieve"][b, :int(ver["n_leaves"][b])]
+        chain = max(([int(x) for x in r if x >= 0] for r in rows), key=len)     # the deepest path
+        d = min(depths[b % len(depths)], len(chain) - 1)
+        for here, nxt in zip(chain[:d], chain[1:d + 1]):
+            out[b, here, int(ver["tokens"][b, nxt])] = 1000.0
+        kids = {int(ver["tokens"][b, i]) for i in range(n) if int(ver["parents"][b, i]) == chain[d]}
+        out[b, chain[d], next(t for t in range(V) if t not in kids)] = 1000.0
+        got.append(d)
+    return out, got
+
+
+def expand_full_level(c2t, dev, weights, root, prefix, stream, dtype=torch.float32, scale: float = 4.0,
+                      reps: int = 20):
+    """Times the expand kernel on full levels of the workload with other logits than the headline's: fp32 instead
+    of bf16, or another temperature scale (levels 1-3, three distinct buffers, so every launch reads from DRAM).
+    Returns None if the frontier does not fill."""
     w = WORKLOAD
     B, V, K, F, N = w["B"], w["V"], w["K"], w["F"], w["N"]
     levels = 4
     w1, b1, w2, b2 = weights
-    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32, max_depth=levels, topk=K, frontier_cap=F, budget=N,
-                     threshold=w["beta"], hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
+    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32 if dtype == torch.float32 else c2t.BF16, max_depth=levels,
+                     topk=K, frontier_cap=F, budget=N, threshold=0.0, classifier=c2t.CLS_IDENTITY_JOINT,
+                     hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
     ctx = c2t.Context(cfg)
-    draft = [c2t_inputs.draft_logits(B, F, V, 0, l, torch.float32, device=dev) for l in range(levels)]
+    draft = [c2t_inputs.draft_logits(B, F, V, 0, l, dtype, scale, device=dev) for l in range(levels)]
     rows = []
     ms = []
     for rep in range(reps + 3):
@@ -453,9 +584,13 @@ def expand_full_level_fp32(c2t, dev, weights, root, prefix, stream, reps: int = 
     torch.cuda.synchronize()
     if min(rows[1:]) != B * F:
         return None
-    us = sum(a.elapsed_time(b) for a, b in ms) / len(ms) * 1e3
-    nbytes = B * F * V * 4
-    return {"rows": B * F, "bytes": nbytes, "us": us, "gbs": nbytes / (us * 1e-6) / 1e9}
+    t = sorted(a.elapsed_time(b) * 1e3 for a, b in ms)
+    us = sum(t) / len(t)
+    nbytes = B * F * V * (4 if dtype == torch.float32 else 2)
+    ctx.close()
+    return {"rows": B * F, "bytes": nbytes, "us": us, "us_median": t[len(t) // 2], "us_min": t[0],
+            "gbs": nbytes / (us * 1e-6) / 1e9, "scale": scale, "dtype": "f32" if dtype == torch.float32 else "bf16",
+            "note": "threshold 0 with the identity classifier, so that every level has B*F active rows"}
 
 
 def single_sequence_latency(c2t, dev, stream, steps: int = 60, sets: int = 4):
@@ -522,6 +657,119 @@ def single_sequence_latency(c2t, dev, stream, steps: int = 60, sets: int = 4):
             print(f"bench.py: CUDA graph replay of the single-sequence case skipped: {exc}", file=sys.stderr)
         ctx.close()
     return out
+
+
+def _time_steps(fn, n, warm=3):
+    for i in range(warm):
+        fn(i)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(n):
+        fn(warm + i)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / n * 1e3
+
+
+def config1_single_sequence_fp32(c2t, dev, stream, steps: int = 120, sets: int = 12):
+    """B=1, V=32000, fp32, D=6, K=F=10, N=60, threshold 0.5: microseconds per decode step.  A step's logits (15 MB)
+    would stay in L2, so the steps rotate over `sets` input sets (185 MB)."""
+    B, V, D, K, F, N, hidden = 1, 32000, 6, 10, 10, 60, 16
+    w1, b1, w2, b2 = make_weights(hidden)
+    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32, max_depth=D, topk=K, frontier_cap=F, budget=N, threshold=0.5,
+                     hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
+    ctx = c2t.Context(cfg)
+    inputs = []
+    for k in range(sets):
+        inputs.append(([c2t_inputs.draft_logits(B, F, V, k, l, torch.float32, device=dev) for l in range(D)],
+                       c2t_inputs.target_logits(B, ctx.Nw, V, k, torch.float32, device=dev),
+                       c2t_inputs.root_tokens(B, V, k).to(dev), c2t_inputs.prefix_lengths(B).to(dev)))
+    nodes, taus = [], []
+    for k in range(sets):
+        ctx.decode_step(*inputs[k], stream=stream)
+        nodes.append(int(ctx.verify["n_nodes"][0])); taus.append(int(ctx.accepted["accept_len"][0]))
+    us = _time_steps(lambda i: ctx.decode_step(*inputs[i % sets], stream=stream), steps)
+    ctx.close()
+    return {"workload": "B=1, V=32000, fp32, depth 6, top-k 10, frontier cap 10, budget 60, threshold 0.5, MLP hidden 16",
+            "l2": f"steps rotate over {sets} input sets (185 MB, larger than L2)", "us_per_step": us,
+            "mean_final_nodes": sum(nodes) / sets, "mean_accept_len": sum(taus) / sets}
+
+
+def config2_chained_steps(c2t, dev, stream, steps: int = 64, sets: int = 16):
+    """B=8, V=32000, bf16, D=8, K=F=10, N=60, threshold 0.5: 64 decode steps in a row, each starting from the
+    previous step's next token and from a prefix that is accept_len + 1 tokens longer (the state stays on the
+    device).  The logits of step s are input set s mod `sets` (16 sets, 1.2 GB)."""
+    B, V, D, K, F, N, hidden = 8, 32000, 8, 10, 10, 60, 16
+    w1, b1, w2, b2 = make_weights(hidden)
+    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.BF16, max_depth=D, topk=K, frontier_cap=F, budget=N, threshold=0.5,
+                     hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
+    ctx = c2t.Context(cfg)
+    inputs = [([c2t_inputs.draft_logits(B, F, V, k, l, torch.bfloat16, device=dev) for l in range(D)],
+               c2t_inputs.target_logits(B, ctx.Nw, V, k, torch.bfloat16, device=dev)) for k in range(sets)]
+    root0 = c2t_inputs.root_tokens(B, V, 0).to(dev)
+    prefix0 = c2t_inputs.prefix_lengths(B).to(dev)
+
+    def chain(record):
+        root, prefix = root0, prefix0
+        for s in range(steps):
+            ctx.decode_step(inputs[s % sets][0], inputs[s % sets][1], root, prefix, stream=stream)
+            if record is not None:
+                record.append((ctx.verify["n_nodes"].clone(), ctx.accepted["accept_len"].clone()))
+            root = ctx.accepted["next_token"].clone()
+            prefix = prefix + ctx.accepted["accept_len"] + 1
+        return prefix
+
+    rec = []
+    chain(rec)                                          # warm-up, and the counts (the chain is deterministic)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    last_prefix = chain(None)
+    b.record()
+    torch.cuda.synchronize()
+    nodes = torch.stack([r[0] for r in rec]).float()
+    taus = torch.stack([r[1] for r in rec]).float()
+    grown = (last_prefix - prefix0).float().mean().item()
+    ctx.close()
+    return {"workload": "B=8, V=32000, bf16, depth 8, top-k 10, frontier cap 10, budget 60, threshold 0.5, 64 chained steps",
+            "us_per_step": a.elapsed_time(b) / steps * 1e3, "steps": steps, "mean_accept_len": taus.mean().item(),
+            "mean_final_nodes": nodes.mean().item(), "mean_tokens_committed_per_sequence": grown}
+
+
+def config5_ablation_sweep(c2t, dev, stream, depth: int = 8, steps: int = 8):
+    """B=32; vocabulary {32000, 128256} x dtype {fp32, bf16} x temperature scale {1, 4, 8} x classifier {identity
+    on the joint probability (EAGLE-2's expand + rerank), the FFN at threshold 0.5} x budget {20, 40, 60, 80} at
+    depth 8: kept candidates, accept length against the synthetic target rows, microseconds per level."""
+    B, K, F, hidden = 32, 10, 10, 16
+    w1, b1, w2, b2 = make_weights(hidden)
+    rows = []
+    for V in (32000, 128256):
+        for dtype in (torch.float32, torch.bfloat16):
+            for scale in (1.0, 4.0, 8.0):
+                draft = [c2t_inputs.draft_logits(B, F, V, 0, l, dtype, scale, device=dev) for l in range(depth)]
+                target = c2t_inputs.target_logits(B, 80, V, 0, dtype, scale, device=dev)
+                root = c2t_inputs.root_tokens(B, V, 0).to(dev)
+                prefix = c2t_inputs.prefix_lengths(B).to(dev)
+                for classifier, beta in ((c2t.CLS_IDENTITY_JOINT, 0.0), (c2t.CLS_MLP, 0.5)):
+                    for N in (20, 40, 60, 80):
+                        cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32 if dtype == torch.float32 else c2t.BF16,
+                                         max_depth=depth, topk=K, frontier_cap=F, budget=N, threshold=beta,
+                                         classifier=classifier, hidden=hidden, w1=w1, b1=b1, w2=w2, b2=b2,
+                                         device=dev.index)
+                        ctx = c2t.Context(cfg)
+                        us = _time_steps(lambda i: ctx.decode_step(draft, target, root, prefix, stream=stream), steps, 2)
+                        view = ctx.c2t_get_view()
+                        rows.append({"V": V, "dtype": "f32" if dtype == torch.float32 else "bf16", "scale": scale,
+                                     "classifier": "identity_joint" if classifier == c2t.CLS_IDENTITY_JOINT else "mlp",
+                                     "budget": N, "mean_tree_nodes_before_rerank": view["tree_n"].float().mean().item(),
+                                     "mean_final_nodes": ctx.verify["n_nodes"].float().mean().item(),
+                                     "mean_accept_len": ctx.accepted["accept_len"].float().mean().item(),
+                                     "us_per_level": us / depth})      # whole step / depth
+                        ctx.close()
+                del draft, target
+    return {"workload": f"B=32, depth {depth}, top-k 10, frontier cap 10; the same step repeated {steps} times "
+                        "(logits of the larger cases exceed L2)", "rows": rows}
 
 
 def run_profile(args) -> None:
