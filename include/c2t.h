@@ -59,6 +59,7 @@ typedef enum { C2T_ADD_FRONTIER = 0, C2T_ADD_ALL_SURVIVORS = 1 } c2t_tree_add;
 #define C2T_ERANGE  (-3)   /* a size exceeds a C2T_MAX_* limit or the workspace is small */
 #define C2T_EORDER  (-4)   /* calls out of sequence within a decode step                 */
 #define C2T_ECUDA   (-5)   /* a CUDA runtime call failed                                 */
+#define C2T_ENOMEM  (-6)   /* the host could not allocate the context                    */
 
 #define C2T_MAX_BATCH     4096
 #define C2T_MAX_TOPK      32
@@ -74,6 +75,10 @@ typedef enum { C2T_ADD_FRONTIER = 0, C2T_ADD_ALL_SURVIVORS = 1 } c2t_tree_add;
 #define C2T_ST_POSINF_LOGIT  2u
 #define C2T_ST_ALL_NEGINF    4u
 #define C2T_ST_TREE_OVERFLOW 8u
+/* The library caught itself outside its own bounds: a row has more partial records than the workspace
+ * was carved for, or (in a build with -DC2T_DEBUG_BOUNDS) an index check failed.  The access is
+ * clamped or skipped, never made; the sequence's results are unspecified.  Never set by data. */
+#define C2T_ST_INTERNAL      16u
 
 /*
  * Method parameters (Alg. 1's inputs d_max and beta; Top-K of Sec. 4.2.2 split into the

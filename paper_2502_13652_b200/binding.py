@@ -14,14 +14,15 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libc2t.so")
+# C2T_LIBRARY selects another build of the same library (the -DC2T_DEBUG_BOUNDS variant, see build.py)
+LIB_PATH = os.environ.get("C2T_LIBRARY") or os.path.join(_HERE, "libc2t.so")
 
 F32, BF16 = 0, 1
 CLS_MLP, CLS_IDENTITY_JOINT, CLS_IDENTITY_COND = 0, 1, 2
 ADD_FRONTIER, ADD_ALL_SURVIVORS = 0, 1
 FINAL = -1
-OK, EINVAL, EALIGN, ERANGE, EORDER, ECUDA = 0, -1, -2, -3, -4, -5
-ST_NAN_LOGIT, ST_POSINF_LOGIT, ST_ALL_NEGINF, ST_TREE_OVERFLOW = 1, 2, 4, 8
+OK, EINVAL, EALIGN, ERANGE, EORDER, ECUDA, ENOMEM = 0, -1, -2, -3, -4, -5, -6
+ST_NAN_LOGIT, ST_POSINF_LOGIT, ST_ALL_NEGINF, ST_TREE_OVERFLOW, ST_INTERNAL = 1, 2, 4, 8, 16
 
 
 class C2TError(RuntimeError):

@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kPassThreads, kPassCtasPerSm) argmax_pass_kern
         unsigned long long other = __shfl_down_sync(kFull, best, o);
         best = other > best ? other : best;
       }
-      if (lane == 0) p.part_best[slot] = best;
+      if (lane == 0 && C2T_IN_BOUNDS(slot, p.n_slots, p.status)) p.part_best[slot] = best;
     }
     __syncthreads();
     pos += seg;

@@ -103,6 +103,7 @@ extern "C" int c2t_row_argmax_static(const void *logits_dev, int32_t rows, int32
   p.V = vocab; p.K = 1; p.B = rows; p.rows_per_seq_max = 1;
   p.counts = pd.scratch->counts;  // address arithmetic on a device pointer, never dereferenced here
   p.max_splits = max_splits;
+  p.n_slots = (int64_t)rows * max_splits;
   p.info = &pd.scratch->info;
   p.part_best = pd.scratch->best;
   if (launch_argmax_pass(p, dtype, pd.grid, s) != cudaSuccess) return C2T_ECUDA;

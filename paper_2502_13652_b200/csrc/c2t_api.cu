@@ -184,7 +184,7 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   }
 
   c2t_ctx *ctx = new (std::nothrow) c2t_ctx;
-  if (!ctx) return C2T_EINVAL;
+  if (!ctx) return C2T_ENOMEM;
   memset(ctx, 0, sizeof *ctx);
   ctx->cfg = *cfg;
   ctx->cfg.w1 = ctx->cfg.b1 = ctx->cfg.w2 = ctx->cfg.b2 = nullptr;
@@ -247,6 +247,8 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   p.V = t.V; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
   p.counts = t.frontier_n[level & 1];
   p.max_splits = t.max_splits;
+  p.n_slots = (int64_t)t.B * t.F * t.max_splits;
+  p.status = t.status;
   p.info = t.info_draft;
   p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
   p.row_off = t.row_off_draft;
@@ -298,6 +300,8 @@ int c2t_expand_level_shard(c2t_ctx *ctx, int level, const void *logits_dev, int6
   p.V = vocab_count; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
   p.counts = t.frontier_n[level & 1];
   p.max_splits = t.max_splits;                    // sized for whole rows: enough for any part of one
+  p.n_slots = (int64_t)t.B * t.F * t.max_splits;
+  p.status = t.status;
   p.info = t.info_draft;
   p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
   p.row_off = t.row_off_draft;
@@ -369,6 +373,8 @@ int c2t_accept(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, 
   p.V = t.V; p.K = 1; p.B = t.B; p.rows_per_seq_max = t.Nw;
   p.counts = t.final_n;
   p.max_splits = t.max_splits_tgt;
+  p.n_slots = (int64_t)t.B * t.Nw * t.max_splits_tgt;
+  p.status = t.status;
   p.info = t.info_target;
   p.part_best = t.part_best;
   if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, (cudaStream_t)stream) != cudaSuccess)
@@ -395,6 +401,8 @@ int c2t_argmax_shard(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_st
   p.V = vocab_count; p.K = 1; p.B = t.B; p.rows_per_seq_max = t.Nw;
   p.counts = t.final_n;
   p.max_splits = t.max_splits_tgt;
+  p.n_slots = (int64_t)t.B * t.Nw * t.max_splits_tgt;
+  p.status = t.status;
   p.info = t.info_target;
   p.part_best = t.part_best;
   if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, (cudaStream_t)stream) != cudaSuccess)
@@ -434,6 +442,8 @@ int c2t_accept_lazy(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_str
   p.counts = t.walk_active;          // one row per sequence that is still walking ...
   p.row_sel = t.walk_cur;            // ... the row of its current node
   p.max_splits = t.max_splits_tgt;
+  p.n_slots = (int64_t)t.B * t.Nw * t.max_splits_tgt;
+  p.status = t.status;
   p.info = t.info_target;
   p.part_best = t.part_best;
   cudaStream_t s = (cudaStream_t)stream;
@@ -451,7 +461,7 @@ int c2t_status(c2t_ctx *ctx, uint32_t *bits_host, uint32_t *per_seq_host, void *
   if (!ctx || !bits_host) return C2T_EINVAL;
   const int B = ctx->cfg.batch;
   uint32_t *tmp = per_seq_host ? per_seq_host : new (std::nothrow) uint32_t[B];
-  if (!tmp) return C2T_EINVAL;
+  if (!tmp) return C2T_ENOMEM;
   cudaError_t e = cudaMemcpyAsync(tmp, ctx->t.status, sizeof(uint32_t) * B, cudaMemcpyDeviceToHost,
                                   (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
@@ -542,6 +552,7 @@ const char *c2t_strerror(int code) {
     case C2T_ERANGE: return "size out of range";
     case C2T_EORDER: return "call out of order";
     case C2T_ECUDA: return "CUDA runtime error";
+    case C2T_ENOMEM: return "out of host memory";
     default: return "unknown error";
   }
 }

@@ -32,6 +32,24 @@ __device__ __forceinline__ int32_t key_token(unsigned long long k) {
 // never produces inf - inf or 0 * inf in the running sums.
 constexpr float kNegInfAsFinite = -1.7e38f;   // anything at or below this was -inf (or as good as)
 
+// ---------------------------------------------------------------- index checks
+// A build with -DC2T_DEBUG_BOUNDS checks the indices of the kernels' writes to shared memory queues, pools and
+// workspace records: a failed check sets C2T_ST_INTERNAL in the given status word (if there is one) and the guarded
+// access is skipped.  It stands in for a memory checker where none can be run.  In a normal build the check is the
+// constant `true`.
+#ifdef __CUDACC__
+#ifdef C2T_DEBUG_BOUNDS
+__device__ __forceinline__ bool c2t_in_bounds(unsigned long long i, unsigned long long n, uint32_t *status) {
+  if (i < n) return true;
+  if (status) atomicOr(status, (uint32_t)C2T_ST_INTERNAL);
+  return false;
+}
+#define C2T_IN_BOUNDS(i, n, status) c2t_in_bounds((unsigned long long)(i), (unsigned long long)(n), (status))
+#else
+#define C2T_IN_BOUNDS(i, n, status) true
+#endif
+#endif
+
 // ---------------------------------------------------------------- launch chain
 // The kernels of a decode step form a chain in which each one consumes what the one before wrote.
 // They are launched with programmatic stream serialisation: the next kernel's CTAs may be placed
@@ -103,6 +121,8 @@ struct PassParams {
   const int32_t *counts;            // [B] active rows per sequence, device
   const int32_t *row_sel;           // arg-max pass only, may be null: [B] the row of sequence b to read (then counts is 0 or 1)
   int32_t max_splits;               // partial slots per row
+  int64_t n_slots;                  // partial slots in the workspace (rows the workspace was carved for x max_splits)
+  uint32_t *status;                 // may be null: a status word for C2T_ST_INTERNAL (the first sequence's)
   PassInfo *info;                   // written by CTA 0
   int32_t *row_off;                 // may be null: [B+1] first active row of every sequence, written by CTA 0
   // expand: per (row, split) partial

@@ -305,7 +305,8 @@ struct Drained {
 // another step might not fit, and at the end, the pool is ranked by counting: the K largest
 // keys stay (sorted, not summed yet), the rest is summed.
 template <bool BF16>
-__device__ __forceinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc acc, float c, float m, float thr) {
+__device__ __forceinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Acc acc, float c, float m, float thr,
+                                               uint32_t *status) {
   constexpr int EPV = Vec<BF16>::N;        // elements per vector
   constexpr int VPS = 32 / EPV;            // vectors per step
   const int lane = threadIdx.x & 31;
@@ -370,7 +371,7 @@ __device__ __forceinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Ac
       else acc_scalar(acc, c, x);                    // (a NaN element poisons the sums, as it must)
     }
     const unsigned mask = __ballot_sync(kFull, cand);
-    if (cand) ws->pool[pn + __popc(mask & lt_mask)] = key;
+    if (cand && C2T_IN_BOUNDS(pn + __popc(mask & lt_mask), kPool, status)) ws->pool[pn + __popc(mask & lt_mask)] = key;
     pn += __popc(mask);
   }
   __syncwarp();
@@ -386,7 +387,7 @@ __device__ __forceinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Ac
 // no lane is past the segment's end.
 template <bool BF16, bool WHOLE>
 __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, SegState &st, int vt, int v1,
-                                              unsigned lt_mask) {
+                                              unsigned lt_mask, uint32_t *status) {
   using VT = Vec<BF16>;
   float vm[kVPL];
 #pragma unroll
@@ -412,8 +413,10 @@ __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, Se
     for (int u = 0; u < kVPL; ++u) {
       if (hit[u]) {
         const int pos = st.qn + __popc(mask[u] & lt_mask);
-        ws->qdata[pos] = g.q[u];
-        ws->qindex[pos] = vt + u * 32;
+        if (C2T_IN_BOUNDS(pos, kQueueCap, status)) {
+          ws->qdata[pos] = g.q[u];
+          ws->qindex[pos] = vt + u * 32;
+        }
       }
       st.qn += __popc(mask[u]);
     }
@@ -424,9 +427,9 @@ __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, Se
 }
 
 template <bool BF16>
-__device__ __forceinline__ void drain_into(WarpShared *ws, SegState &st, int K) {
+__device__ __forceinline__ void drain_into(WarpShared *ws, SegState &st, int K, uint32_t *status) {
   __syncwarp();                                      // the queue was written by other lanes
-  const Drained d = drain_queue<BF16>(ws, st.qn, K, st.acc, st.c, st.m, st.thr);
+  const Drained d = drain_queue<BF16>(ws, st.qn, K, st.acc, st.c, st.m, st.thr, status);
   st.acc = d.acc; st.c = d.c; st.m = d.m; st.thr = d.thr;
   st.qn = 0;
   __syncwarp();
@@ -506,7 +509,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
         const uint4 *src = reinterpret_cast<const uint4 *>(seg.row) + pre.tv0 + lane;
         int vt = cur.tv0 + lane;
         for (int i = 0; i < k; ++i) {
-          process_group<BF16, true>(ws, g, st, vt, 0, lt_mask);
+          process_group<BF16, true>(ws, g, st, vt, 0, lt_mask, p.status);
           n = next_slot(n);
           vt += kGroupVecs;
           cp_async_wait<kRingSlots - 1>();
@@ -519,7 +522,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
           LaneCopies<kVPL>::all(dst, src);
           cp_async_commit();
           src += kGroupVecs;
-          if (st.qn > kDrainAt) drain_into<BF16>(ws, st, K);
+          if (st.qn > kDrainAt) drain_into<BF16>(ws, st, K, p.status);
         }
         cur.tv0 += k * kGroupVecs;
         pre.tv0 += (k - 1) * kGroupVecs;             // the last step may leave the segment
@@ -528,7 +531,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
     }
     // ---- one group near the end of a segment, everything checked
     const int vt = cur.tv0 + lane;
-    process_group<BF16, false>(ws, g, st, vt, seg.v1, lt_mask);
+    process_group<BF16, false>(ws, g, st, vt, seg.v1, lt_mask, p.status);
     const bool last = cur.last_of_segment();
     cur.advance(p, s_off, esz);
     n = next_slot(n);
@@ -539,7 +542,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       prefetch_group(pre, slot, v_full, lane);
       pre.advance(p, s_off, esz);
     }
-    if (last || st.qn > kDrainAt) drain_into<BF16>(ws, st, K);
+    if (last || st.qn > kDrainAt) drain_into<BF16>(ws, st, K, p.status);
     if (last) {
       // ---- the segment's record: the K largest keys but the first join the sums; sums in a
       // fixed order, the sorted keys, the held-out head
@@ -554,8 +557,9 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
       const long long split = worker - div_floor((long long)seg.a * vrow + kSegmentPad, span);   // workers before the row's first
       const size_t slot_id = (size_t)seg.a * p.max_splits + (size_t)split;
       const unsigned have = __ballot_sync(kFull, mine != 0ull);
-      if (lane < K) p.part_keys[slot_id * K + lane] = mine;
-      if (lane == 0) {
+      const bool slot_ok = C2T_IN_BOUNDS(slot_id, p.n_slots, p.status);
+      if (lane < K && slot_ok) p.part_keys[slot_id * K + lane] = mine;
+      if (lane == 0 && slot_ok) {
         p.part_held[slot_id] = mine;
         p.part_stats[slot_id] = make_float4(st.c, S, U, __int_as_float(__popc(have)));
       }

@@ -89,7 +89,7 @@ struct RowMerge {
 // best (logit, token) pairs go to out_x / out_tok (shared or global memory, best first, padded with
 // -inf / -1), token ids offset by tok_base; vloc is the length of the rows the pass read (tokens at
 // or past it pad a ragged last vector).  sk: the warp's staging area of kStageKeys keys.
-__device__ RowMerge merge_row_partials(const TreeState &t, const PassInfo &info, int a, int K, int vloc,
+__device__ RowMerge merge_row_partials(const TreeState &t, const PassInfo &info, int seq, int a, int K, int vloc,
                                        unsigned long long *sk, float *out_x, int *out_tok, int tok_base) {
   const int lane = threadIdx.x & 31;
   // the workers that hold a piece of this row: the rows, each behind info.pad virtual vectors, were cut every info.span
@@ -97,7 +97,10 @@ __device__ RowMerge merge_row_partials(const TreeState &t, const PassInfo &info,
   const int c_first = (int)(first_vec / info.span);
   const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
   int n_splits = c_last - c_first + 1;
-  if (n_splits > t.max_splits) n_splits = t.max_splits;
+  if (n_splits > t.max_splits) {                    // the host's sizing and the pass disagree: say so, stay in bounds
+    n_splits = t.max_splits;
+    if (lane == 0) atomicOr(&t.status[seq], C2T_ST_INTERNAL);
+  }
   const size_t slot0 = (size_t)a * t.max_splits;
   const int n_keys = n_splits * K;
 
@@ -278,7 +281,7 @@ __global__ void __launch_bounds__(kTreeThreads) export_rows_kernel(TreeState t, 
   n = n < 0 ? 0 : (n > t.F ? t.F : n);
   for (int j = warp; j < n; j += kTreeWarps) {
     c2t_row_record *r = out + (size_t)b * t.F + j;
-    const RowMerge m = merge_row_partials(t, info, row_off + j, t.K, vloc, s_keys[warp], r->x, r->tok, tok_base);
+    const RowMerge m = merge_row_partials(t, info, b, row_off + j, t.K, vloc, s_keys[warp], r->x, r->tok, tok_base);
     if (lane == 0) {
       r->M = m.M; r->S = m.S; r->T = m.T;
       r->n = m.n_valid;
@@ -340,7 +343,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     uint32_t shard_faults = 0u;
     const RowMerge m = records
         ? merge_row_records(t, records, n_shards, b, j, K, &s_x[j * K], &s_tok[j * K], &shard_faults)
-        : merge_row_partials(t, info, row_off + j, K, t.V, s_keys[warp], &s_x[j * K], &s_tok[j * K], 0);
+        : merge_row_partials(t, info, b, row_off + j, K, t.V, s_keys[warp], &s_x[j * K], &s_tok[j * K], 0);
     if (lane == 0) {
       const uint32_t fault = shard_faults ? shard_faults : row_fault_bits(m.top, m.S, m.T);
       const double L = log1p(m.S);                // ln sum_v e^(x_v - M); the maximum contributes the 1
@@ -444,6 +447,7 @@ __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, 
     }
     if (s_sel[c] && !overflow) {
       const int slot = off_sel++;
+      if (!C2T_IN_BOUNDS(slot, F, &t.status[b])) continue;
       t.frontier_node[nxt][(size_t)b * F + slot] = id;
       if (out.token) out.token[(size_t)b * F + slot] = s_tok[c];
       if (out.node_id) out.node_id[(size_t)b * F + slot] = id;
@@ -577,12 +581,15 @@ __global__ void __launch_bounds__(kTreeThreads) build_verify_kernel(TreeState t,
 // ---------------------------------------------------------------- accept ----
 
 // best key of active row `a` of the last arg-max pass (0: none)
-__device__ __forceinline__ unsigned long long row_best_key(const TreeState &t, const PassInfo &info, int a) {
+__device__ __forceinline__ unsigned long long row_best_key(const TreeState &t, const PassInfo &info, int seq, int a) {
   const long long first_vec = (long long)a * info.vec_per_row;
   const int c_first = (int)(first_vec / info.span);
   const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
   int n_splits = c_last - c_first + 1;
-  if (n_splits > t.max_splits_tgt) n_splits = t.max_splits_tgt;
+  if (n_splits > t.max_splits_tgt) {
+    n_splits = t.max_splits_tgt;
+    atomicOr(&t.status[seq], C2T_ST_INTERNAL);
+  }
   unsigned long long best = 0ull;
   for (int s = 0; s < n_splits; ++s) {
     unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + s];
@@ -616,7 +623,7 @@ __global__ void __launch_bounds__(kTreeThreads) export_best_kernel(TreeState t, 
   for (int i = threadIdx.x; i < Nw; i += kTreeThreads) {
     unsigned long long key = 0ull;
     if (i < n) {
-      const unsigned long long best = row_best_key(t, info, row_off + i);
+      const unsigned long long best = row_best_key(t, info, b, row_off + i);
       if (best) key = (best & 0xFFFFFFFF00000000ull) | (0xFFFFFFFFu - (uint32_t)(key_token(best) + tok_base));
     }
     out[(size_t)b * Nw + i] = key;
@@ -658,7 +665,7 @@ __global__ void __launch_bounds__(kTreeThreads) accept_walk_kernel(TreeState t, 
           best = k > best ? k : best;
         }
       } else {
-        best = row_best_key(t, info, row_off + i);
+        best = row_best_key(t, info, b, row_off + i);
       }
       tok = best ? key_token(best) : -1;
     }
@@ -782,7 +789,10 @@ __global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState
     const int c_first = (int)(first_vec / info.span);
     const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
     int n_splits = c_last - c_first + 1;
-    if (n_splits > t.max_splits_tgt) n_splits = t.max_splits_tgt;
+    if (n_splits > t.max_splits_tgt) {
+      n_splits = t.max_splits_tgt;
+      atomicOr(&t.status[b], C2T_ST_INTERNAL);
+    }
     unsigned long long best = 0ull;
     for (int sp = 0; sp < n_splits; ++sp) {
       const unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + sp];

@@ -32,30 +32,49 @@ def shard_ranges(vocab: int, world: int, elem_bytes: int) -> List[Tuple[int, int
     return out
 
 
-def gather_row_records(local: torch.Tensor, group: Optional[dist.ProcessGroup] = None) -> torch.Tensor:
+def gather_row_records(local: torch.Tensor, group: Optional[dist.ProcessGroup] = None,
+                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """All-gathers one rank's records [B, F, bytes] into [world, B, F, bytes], shard-major in rank order
-    (= ascending token order when the ranges come from `shard_ranges`)."""
+    (= ascending token order when the ranges come from `shard_ranges`).  `out`: a buffer of that shape to
+    gather into (allocated if absent)."""
     world = dist.get_world_size(group)
-    out = torch.empty((world * local.shape[0],) + tuple(local.shape[1:]), dtype=local.dtype, device=local.device)
-    dist.all_gather_into_tensor(out, local.contiguous(), group=group)      # concatenated along the first dimension
-    return out.view((world,) + tuple(local.shape))
+    if out is None:
+        out = torch.empty((world,) + tuple(local.shape), dtype=local.dtype, device=local.device)
+    assert out.is_contiguous() and tuple(out.shape) == (world,) + tuple(local.shape)
+    dist.all_gather_into_tensor(out.view((world * local.shape[0],) + tuple(local.shape[1:])), local.contiguous(),
+                                group=group)                               # concatenated along the first dimension
+    return out
+
+
+class ExchangeBuffers:
+    """The buffers of the exchange, allocated once per context and process group, so that a level allocates nothing."""
+
+    def __init__(self, ctx, group: Optional[dist.ProcessGroup] = None):
+        world = dist.get_world_size(group)
+        self.records = ctx.new_row_records(world)                      # [world, B, F, bytes]
+        self.local = ctx.new_row_records(1)[0]                         # [B, F, bytes]
+        self.keys = torch.zeros((world, ctx.B, ctx.Nw), dtype=torch.int64, device=self.records.device)
+        self.local_keys = torch.zeros((ctx.B, ctx.Nw), dtype=torch.int64, device=self.records.device)
 
 
 def vocab_parallel_level(ctx, level: int, shard_logits: torch.Tensor, vocab_begin: int,
-                         group: Optional[dist.ProcessGroup] = None, stream=None) -> None:
+                         group: Optional[dist.ProcessGroup] = None, stream=None,
+                         buffers: Optional[ExchangeBuffers] = None) -> None:
     """One level of the tree on this rank: `shard_logits` [B, F, count] are this rank's token range
-    starting at `vocab_begin`.  The collective runs on the current stream, after the export."""
-    local = ctx.new_row_records(1)[0]
+    starting at `vocab_begin`.  The collective runs on the current stream, after the export.  Pass the
+    `ExchangeBuffers` of the context to keep allocations off this path."""
+    buffers = buffers or ExchangeBuffers(ctx, group)
     ctx.c2t_expand_level_shard(level, shard_logits, stream)
-    ctx.c2t_export_row_records(level, vocab_begin, local, stream)
-    records = gather_row_records(local, group)
+    ctx.c2t_export_row_records(level, vocab_begin, buffers.local, stream)
+    records = gather_row_records(buffers.local, group, buffers.records)
     ctx.c2t_prune_gathered(level, records, stream)
 
 
 def vocab_parallel_accept(ctx, target_shard: torch.Tensor, vocab_begin: int,
-                          group: Optional[dist.ProcessGroup] = None, stream=None) -> None:
+                          group: Optional[dist.ProcessGroup] = None, stream=None,
+                          buffers: Optional[ExchangeBuffers] = None) -> None:
     """The acceptance walk with sharded target logits: this rank's best key per final node, one all-gather of
     8 bytes per node, the walk on every rank."""
-    local = torch.zeros((ctx.B, ctx.Nw), dtype=torch.int64, device=target_shard.device)
-    ctx.c2t_argmax_shard(target_shard, vocab_begin, local, stream)
-    ctx.c2t_accept_gathered(gather_row_records(local, group), stream)
+    buffers = buffers or ExchangeBuffers(ctx, group)
+    ctx.c2t_argmax_shard(target_shard, vocab_begin, buffers.local_keys, stream)
+    ctx.c2t_accept_gathered(gather_row_records(buffers.local_keys, group, buffers.keys), stream)

@@ -106,8 +106,8 @@ def test_null_context_is_rejected(L):
 
 def test_strerror(L):
     assert L.c2t_strerror(0) == b"ok"
-    seen = {L.c2t_strerror(code) for code in (0, -1, -2, -3, -4, -5)}
-    assert len(seen) == 6
+    seen = {L.c2t_strerror(code) for code in (0, -1, -2, -3, -4, -5, -6)}
+    assert len(seen) == 7
     assert L.c2t_strerror(-99) == b"unknown error"
 
 
