@@ -69,6 +69,7 @@ typedef enum { C2T_ADD_FRONTIER = 0, C2T_ADD_ALL_SURVIVORS = 1 } c2t_tree_add;
 #define C2T_MAX_BUDGET    1024
 #define C2T_MAX_TREE      8192   /* nodes per sequence before the Top-N rerank */
 #define C2T_MAX_SHARDS    32     /* vocabulary shards merged by c2t_prune_gathered */
+#define C2T_FUSED_MAX_BATCH 2    /* largest batch for which c2t_expand_prune_level uses a single launch */
 
 /* per-sequence status bits */
 #define C2T_ST_NAN_LOGIT     1u
@@ -166,6 +167,18 @@ typedef struct {
  *   last level pruned (any number of levels <= D).
  */
 int c2t_prune(c2t_ctx *ctx, int level, const c2t_frontier *out, void *stream);
+
+/*
+ * c2t_expand_level(level, ...) followed by c2t_prune(level, out), as one call (Sec. 4.2.1, Eq. 1-2, Eq. 4,
+ * Alg. 1, Sec. 4.2.2: the same operations, the same results bit for bit).  For batches of at most
+ * C2T_FUSED_MAX_BATCH sequences (the paper's own operating point is one sequence) it is ONE kernel launch:
+ * the thread block that finishes the vocabulary pass last does the per-sequence work, which halves the
+ * launch-to-launch latency that bounds such a step.  Larger batches, and contexts with entropy_top_m > 0,
+ * get the two (or three) launches of the separate calls.  Arguments, alignment rules and errors as for
+ * c2t_expand_level; `out` as for c2t_prune (may be NULL).
+ */
+int c2t_expand_prune_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t seq_stride,
+                           int64_t row_stride, const c2t_frontier *out, void *stream);
 
 /* Verification inputs, written by c2t_build_verify.  Caller-owned device arrays, NULL = skip.
  * Nw = c2t_final_width, W = c2t_mask_words, D = cfg.max_depth. */

@@ -113,6 +113,9 @@ def lib() -> C.CDLL:
         L.c2t_begin_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.c2t_expand_level.restype = C.c_int
         L.c2t_expand_level.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p]
+        L.c2t_expand_prune_level.restype = C.c_int
+        L.c2t_expand_prune_level.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int64,
+                                             P(c2t_frontier), C.c_void_p]
         L.c2t_prune.restype = C.c_int
         L.c2t_prune.argtypes = [C.c_void_p, C.c_int, P(c2t_frontier), C.c_void_p]
         L.c2t_expand_level_shard.restype = C.c_int
@@ -311,6 +314,14 @@ class Context:
         _check(lib().c2t_expand_level(self._h, level, logits.data_ptr(), logits.stride(0), logits.stride(1),
                                       _stream(stream)), "c2t_expand_level")
 
+    def c2t_expand_prune_level(self, level: int, logits: torch.Tensor, stream=None, emit: bool = True) -> None:
+        """c2t_expand_level and c2t_prune of a level as one call (one launch for batches of at most 2 sequences)."""
+        assert logits.is_cuda and logits.dtype == self.cfg.torch_dtype and logits.dim() == 3
+        assert logits.shape[0] == self.B and logits.shape[2] == self.V and logits.stride(2) == 1
+        out = C.byref(self._frontier_c) if emit else None
+        _check(lib().c2t_expand_prune_level(self._h, level, logits.data_ptr(), logits.stride(0), logits.stride(1), out,
+                                            _stream(stream)), "c2t_expand_prune_level")
+
     def c2t_prune(self, level: int, stream=None, emit: bool = True) -> None:
         out = C.byref(self._frontier_c) if (emit and level != FINAL) else None
         _check(lib().c2t_prune(self._h, level, out, _stream(stream)), "c2t_prune")
@@ -458,8 +469,7 @@ class Context:
                     root_tok: torch.Tensor, prefix_len: torch.Tensor, stream=None) -> None:
         self.c2t_begin_step(root_tok, prefix_len, stream)
         for level in range(self.D):
-            self.c2t_expand_level(level, draft_levels[level], stream)
-            self.c2t_prune(level, stream)
+            self.c2t_expand_prune_level(level, draft_levels[level], stream)
         self.c2t_prune(FINAL, stream)
         self.c2t_build_verify(stream)
         self.c2t_accept(target, stream)

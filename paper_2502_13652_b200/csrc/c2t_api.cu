@@ -117,6 +117,7 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   s.walk_cur = w.take<int32_t>(B);
   s.walk_len = w.take<int32_t>(B);
   s.status = w.take<uint32_t>(B);
+  s.ticket = w.take<uint32_t>(1);
   s.info_draft = w.take<PassInfo>(1);
   s.info_target = w.take<PassInfo>(1);
   s.row_off_draft = w.take<int32_t>(B + 1);
@@ -211,6 +212,7 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
     if (e == cudaSuccess) e = cudaMemcpy(t.b2, cfg->b2, sizeof(float), cudaMemcpyHostToDevice);
   }
   if (e == cudaSuccess) e = cudaMemset(t.status, 0, sizeof(uint32_t) * cfg->batch);
+  if (e == cudaSuccess) e = cudaMemset(t.ticket, 0, sizeof(uint32_t));
   if (e != cudaSuccess) { cudaGetLastError(); delete ctx; return C2T_ECUDA; }
   *out = ctx;
   return C2T_OK;
@@ -279,6 +281,38 @@ int c2t_prune(c2t_ctx *ctx, int level, const c2t_frontier *out, void *stream) {
   if (launch_prune_level(ctx->t, level, out, nullptr, 0, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
   ctx->launches += 1;
   ctx->expanded = 0;
+  ctx->next_level = level + 1;
+  return C2T_OK;
+}
+
+int c2t_expand_prune_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t seq_stride, int64_t row_stride,
+                           const c2t_frontier *out, void *stream) {
+  if (!ctx || !logits_dev) return C2T_EINVAL;
+  const TreeState &t = ctx->t;
+  if (t.B > C2T_FUSED_MAX_BATCH || (t.entropy_top_m > 0 && t.entropy_top_m < t.V)) {
+    const int rc = c2t_expand_level(ctx, level, logits_dev, seq_stride, row_stride, stream);
+    return rc != C2T_OK ? rc : c2t_prune(ctx, level, out, stream);
+  }
+  if (!ctx->started || ctx->finalized || ctx->expanded || ctx->shard_expanded || level != ctx->next_level ||
+      level >= ctx->cfg.max_depth)
+    return C2T_EORDER;
+  if (seq_stride < 0 || row_stride < ctx->cfg.vocab) return C2T_EINVAL;
+  if (!aligned16(logits_dev) || (seq_stride * ctx->elem_bytes) % 16 || (row_stride * ctx->elem_bytes) % 16)
+    return C2T_EALIGN;
+  PassParams p;
+  memset(&p, 0, sizeof p);
+  p.logits = logits_dev; p.seq_stride = seq_stride; p.row_stride = row_stride;
+  p.V = t.V; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
+  p.counts = t.frontier_n[level & 1];
+  p.max_splits = t.max_splits;
+  p.n_slots = (int64_t)t.B * t.F * t.max_splits;
+  p.status = t.status;
+  p.info = t.info_draft;
+  p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
+  p.row_off = t.row_off_draft;
+  if (launch_expand_prune(p, t, level, out, ctx->cfg.dtype, ctx->grid_expand, (cudaStream_t)stream) != cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 1;
   ctx->next_level = level + 1;
   return C2T_OK;
 }

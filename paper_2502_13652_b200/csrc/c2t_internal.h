@@ -139,6 +139,10 @@ int max_splits_for(int vocab, int elem_bytes, int workers, int pad);
 cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
 cudaError_t launch_argmax_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
+struct TreeState;
+// expand and prune of a level in one launch (batches of at most C2T_FUSED_MAX_BATCH sequences)
+cudaError_t launch_expand_prune(const PassParams &p, const TreeState &t, int level, const c2t_frontier *out, int dtype,
+                                int grid, cudaStream_t s);
 // ---------------------------------------------------------------- tree state -
 
 struct TreeState {
@@ -165,6 +169,7 @@ struct TreeState {
   int32_t entropy_top_m;       // M of Eq. 3 (0: exact entropy)
   double2 *topm;               // [B, F] {S_M, T_M} of the last expand call when M > 0
   uint32_t *status;            // [B]
+  uint32_t *ticket;            // one counter: CTAs of a fused expand + prune launch that have finished (0 between launches)
   PassInfo *info_draft, *info_target;
   int32_t *row_off_draft;          // [B+1] first row of every sequence in the last expand pass
   float4 *part_stats;

@@ -39,6 +39,7 @@
 // Everything depends only on the warp's own data in a fixed order, so the results are
 // reproducible bit for bit.
 #include "vocab_common.cuh"
+#include "level_prune.cuh"
 
 namespace c2t {
 namespace {
@@ -437,16 +438,15 @@ __device__ __forceinline__ void drain_into(WarpShared *ws, SegState &st, int K, 
 
 // ---------------------------------------------------------------- the kernel
 
+// The pass itself: what every warp of the grid does (a warp returns when its span is done).
 template <bool BF16>
-__global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_kernel(PassParams p) {
+__device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned char *s_dyn) {
   using VT = Vec<BF16>;
-  extern __shared__ __align__(16) unsigned char s_dyn[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   WarpShared *ws = reinterpret_cast<WarpShared *>(s_dyn) + warp;
   int *s_off = reinterpret_cast<int *>(s_dyn + kEWarps * sizeof(WarpShared));
 
   const int K = p.K;
-  chain_enter();
   const int n_rows = build_row_offsets(p.counts, p.B, p.rows_per_seq_max, s_off);   // the only barriers
   if (blockIdx.x == 0 && p.row_off)                  // the pruning kernel finds a sequence's rows with this
     for (int i = threadIdx.x; i <= p.B; i += kExpandThreads) p.row_off[i] = s_off[i];
@@ -571,6 +571,36 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_
   cp_async_wait<0>();
 }
 
+template <bool BF16>
+__global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_kernel(PassParams p) {
+  extern __shared__ __align__(16) unsigned char s_dyn[];
+  chain_enter();
+  expand_pass_body<BF16>(p, s_dyn);
+}
+
+// Expand and prune of a level in one launch, for small batches: the CTA that finishes last (an atomic ticket, nobody
+// waits) has every row's partial records in front of it and does the per-sequence work of c2t_prune for all
+// sequences, one after the other.
+template <bool BF16>
+__global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_prune_kernel(PassParams p, TreeState t, int level,
+                                                                                        c2t_frontier out) {
+  extern __shared__ __align__(16) unsigned char s_dyn[];
+  __shared__ unsigned s_ticket;
+  chain_enter();
+  expand_pass_body<BF16>(p, s_dyn);
+  __threadfence();                                   // this CTA's records, before its ticket
+  __syncthreads();
+  if (threadIdx.x == 0) s_ticket = atomicAdd(t.ticket, 1u);
+  __syncthreads();
+  if (s_ticket != gridDim.x - 1) return;
+  __threadfence();                                   // the other CTAs' records, after their tickets
+  if (threadIdx.x == 0) *t.ticket = 0u;              // for the next launch
+  // the pass's shared memory is free now
+  static_assert(sizeof(PruneShared<kEWarps>) <= kEWarps * sizeof(WarpShared), "the prune's scratch must fit the warps' areas");
+  PruneShared<kEWarps> &sh = *reinterpret_cast<PruneShared<kEWarps> *>(s_dyn);
+  for (int b = 0; b < t.B; ++b) prune_level_body<kExpandThreads, false>(t, level, out, nullptr, 0, b, sh);
+}
+
 }  // namespace
 
 int max_splits_for(int vocab, int elem_bytes, int workers, int pad) {
@@ -587,9 +617,22 @@ static size_t expand_dynamic_smem(int B) {
 
 cudaError_t prepare_expand_pass() {
   const int bytes = (int)expand_dynamic_smem(C2T_MAX_BATCH);
+  const int fused = (int)expand_dynamic_smem(C2T_FUSED_MAX_BATCH);
   cudaError_t e = cudaFuncSetAttribute(expand_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(expand_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_prune_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, fused);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_prune_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, fused);
+  return e;
+}
+
+cudaError_t launch_expand_prune(const PassParams &p, const TreeState &t, int level, const c2t_frontier *out, int dtype,
+                                int grid, cudaStream_t s) {
+  c2t_frontier o = {nullptr, nullptr, nullptr, nullptr};
+  if (out) o = *out;
+  const size_t smem = expand_dynamic_smem(p.B);
+  if (dtype == C2T_BF16)
+    return launch_chained(expand_prune_kernel<true>, dim3(grid), dim3(kExpandThreads), smem, s, p, t, level, o);
+  return launch_chained(expand_prune_kernel<false>, dim3(grid), dim3(kExpandThreads), smem, s, p, t, level, o);
 }
 
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s) {

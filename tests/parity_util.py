@@ -202,7 +202,7 @@ def _excuse_budget(tree, ft, g_src) -> str | None:
 
 
 def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, ctx=None,
-                    draft_dev=None, target_dev=None, shards=None, allow_diverged=0, allow_kinds=()) -> Report:
+                    draft_dev=None, target_dev=None, shards=None, allow_diverged=0, allow_kinds=(), fused=False) -> Report:
     """Runs one decode step on the GPU (level by level) and on the oracle; asserts parity.
 
     shards: token ranges [(begin, end), ...] covering the vocabulary in ascending order.  Every level
@@ -212,6 +212,8 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
 
     draft_cpu: list of D tensors [B,F,V] on CPU (or None when `seqs` rows are pulled from
     draft_dev); seqs: sequences the oracle checks (default all).
+
+    fused: every level through c2t_expand_prune_level (one launch for small batches) instead of the two calls.
 
     allow_diverged / allow_kinds: how many sequences may differ from the oracle through a boundary
     case of the module docstring, and of which kinds; more, or another kind, fails."""
@@ -256,6 +258,8 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
                 ctx.c2t_expand_level_shard(l, draft_dev[l][:, :, v0:v1])
                 ctx.c2t_export_row_records(l, v0, records[g])
             ctx.c2t_prune_gathered(l, records)
+        elif fused:
+            ctx.c2t_expand_prune_level(l, draft_dev[l])
         else:
             ctx.c2t_expand_level(l, draft_dev[l])
             ctx.c2t_prune(l)

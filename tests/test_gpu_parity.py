@@ -26,14 +26,14 @@ def _built():
     assert os.path.exists(c2t.LIB_PATH)
 
 
-def case(B, V, D, K, F, N, beta, dtype, step=0, scale=4.0, allow_diverged=0, allow_kinds=(), **kw):
+def case(B, V, D, K, F, N, beta, dtype, step=0, scale=4.0, allow_diverged=0, allow_kinds=(), fused=False, **kw):
     """One decode step of seeded inputs on both sides.  No sequence may differ from the oracle unless the
     caller names the boundary case and bounds the count (see parity_util)."""
     ocfg, gcfg = make_configs(B, V, D, K, F, N, beta, dtype, **kw)
     Nw = c2t.c2t_final_width(gcfg)
     draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, dtype, step=step, scale=scale)
     rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, allow_diverged=allow_diverged,
-                          allow_kinds=allow_kinds)
+                          allow_kinds=allow_kinds, fused=fused)
     print(f"\n  [{B}x{V} {str(dtype)[6:]} D{D} K{K} F{F} N{N} b{beta}] {rep.line()}")
     assert rep.status_bits == 0
     assert rep.kept_nodes == rep.oracle_kept_nodes or rep.diverged_sequences
@@ -72,6 +72,58 @@ def test_tiny_hand_enumerated_tree():
 
 def test_config1_single_sequence_fp32():
     case(1, 32000, 6, 10, 10, 60, 0.5, torch.float32)
+
+
+@pytest.mark.parametrize("B,V,dtype", [(1, 32000, torch.float32), (2, 32000, torch.bfloat16), (1, 128256, torch.bfloat16),
+                                       (2, 5000, torch.float32)])
+def test_fused_expand_prune_level_against_oracle(B, V, dtype):
+    """Expand and prune of a level in one launch (batches of one or two sequences): against the oracle like the
+    separate calls, and one launch per level."""
+    D = 6
+    ocfg, gcfg = make_configs(B, V, D, 8, 16, 50, 0.4, dtype)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, 16, Nw, dtype)
+    ctx = c2t.Context(gcfg)
+    n0 = ctx.c2t_launch_count()
+    rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, ctx=ctx, fused=True)
+    assert rep.status_bits == 0
+    # begin_step, D fused levels, rerank, verify inputs; then the acceptance calls of the comparison
+    ctx.decode_step([t.cuda() for t in draft], target.cuda(), root.cuda(), prefix.cuda())
+    n1 = ctx.c2t_launch_count()
+    ctx.decode_step([t.cuda() for t in draft], target.cuda(), root.cuda(), prefix.cuda())
+    assert ctx.c2t_launch_count() - n1 == 1 + D + 1 + 1 + 2
+    ctx.close()
+
+
+def test_fused_and_separate_calls_agree_bit_for_bit():
+    B, V, D, K, F, N = 2, 128256, 10, 8, 16, 80
+    _, gcfg = make_configs(B, V, D, K, F, N, 0.3, torch.bfloat16)
+    Nw = c2t.c2t_final_width(gcfg)
+    draft, target, root, prefix = gen_inputs(B, V, D, F, Nw, torch.bfloat16)
+    draft = [t.cuda() for t in draft]; target = target.cuda(); root = root.cuda(); prefix = prefix.cuda()
+    ctx = c2t.Context(gcfg)
+    snaps = []
+    for fused in (False, True, True):
+        ctx.c2t_begin_step(root, prefix)
+        for l in range(D):
+            if fused:
+                ctx.c2t_expand_prune_level(l, draft[l])
+            else:
+                ctx.c2t_expand_level(l, draft[l]); ctx.c2t_prune(l)
+        ctx.c2t_prune(c2t.FINAL); ctx.c2t_build_verify(); ctx.c2t_accept(target)
+        torch.cuda.synchronize()
+        v = ctx.c2t_get_view()
+        n = v["tree_n"].clone()
+        live = torch.arange(ctx.cap, device="cuda")[None, :] < n[:, None]
+        snaps.append([n, torch.where(live, v["tree_token"], 0), torch.where(live, v["tree_parent"], 0),
+                      torch.where(live, v["tree_logP"], 0.0), torch.where(live, v["tree_C"], 0.0),
+                      v["cand_flags"].clone(), ctx.frontier["count"].clone(), ctx.frontier["token"].clone(),
+                      ctx.verify["mask_bits"].clone(), ctx.verify["retrieve"].clone(), ctx.accepted["path"].clone()])
+    assert int(snaps[0][0].max()) > 1
+    for other in snaps[1:]:
+        for a, b in zip(snaps[0], other):
+            assert torch.equal(a, b)
+    ctx.close()
 
 
 def test_config2_batch8_bf16_several_steps():
