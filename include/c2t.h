@@ -320,6 +320,30 @@ int c2t_accept_lazy(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_str
                     int64_t row_stride, const c2t_accept_out *out, void *stream);
 
 /*
+ * c2t_accept_lazy for target logits that are sharded over the vocabulary (Sec. 5 Metrics; the rows read are
+ * still only those on the accepted path).  Every rank drives the same loop:
+ *
+ *   c2t_lazy_begin(out)                                    puts every sequence on its root
+ *   for round = 1 .. D + 1:
+ *     c2t_lazy_argmax_shard(target shard, ..., keys)       this rank's best key of every walking sequence's
+ *                                                          current row, token ids made global ([B] keys, 0 for
+ *                                                          a sequence that has stopped)
+ *     [all-gather of the B keys, 8 bytes per sequence]
+ *     c2t_lazy_step_gathered(round, gathered keys [n_shards, B], n_shards, out)
+ *                                                          largest key per sequence (equal logits: the lower
+ *                                                          token id), then one step of every walk
+ *
+ * A path has at most D + 1 nodes, so D + 1 rounds always finish the walk; rounds after a sequence has
+ * stopped read nothing of it.  `out` as for c2t_accept; results equal c2t_accept's.  Must follow
+ * c2t_prune(C2T_FINAL).  keys_dev: caller-owned device buffers.
+ */
+int c2t_lazy_begin(c2t_ctx *ctx, const c2t_accept_out *out, void *stream);
+int c2t_lazy_argmax_shard(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, int64_t row_stride,
+                          int32_t vocab_count, int32_t vocab_begin, uint64_t *keys_dev, void *stream);
+int c2t_lazy_step_gathered(c2t_ctx *ctx, int round, const uint64_t *keys_dev, int32_t n_shards,
+                           const c2t_accept_out *out, void *stream);
+
+/*
  * The paper has no counterpart to this call; it exists for callers that cannot allocate.
  *
  * Some users of this library may not call cudaMalloc, and may not ask an allocator for a

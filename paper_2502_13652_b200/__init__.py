@@ -12,4 +12,6 @@ from .binding import (  # noqa: F401
     ST_NAN_LOGIT, ST_POSINF_LOGIT, ST_ALL_NEGINF, ST_TREE_OVERFLOW, ST_INTERNAL,
 )
 from .weights import save_classifier, load_classifier  # noqa: F401,E402
-from .vocab_parallel import shard_ranges, gather_row_records, vocab_parallel_level, vocab_parallel_accept  # noqa: F401,E402
+from .vocab_parallel import (  # noqa: F401,E402
+    shard_ranges, gather_row_records, vocab_parallel_level, vocab_parallel_accept, vocab_parallel_accept_lazy,
+    ExchangeBuffers)

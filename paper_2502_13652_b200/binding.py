@@ -118,6 +118,14 @@ def lib() -> C.CDLL:
                                              P(c2t_frontier), C.c_void_p]
         L.c2t_prune.restype = C.c_int
         L.c2t_prune.argtypes = [C.c_void_p, C.c_int, P(c2t_frontier), C.c_void_p]
+        L.c2t_lazy_begin.restype = C.c_int
+        L.c2t_lazy_begin.argtypes = [C.c_void_p, P(c2t_accept_out), C.c_void_p]
+        L.c2t_lazy_argmax_shard.restype = C.c_int
+        L.c2t_lazy_argmax_shard.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
+                                            C.c_void_p, C.c_void_p]
+        L.c2t_lazy_step_gathered.restype = C.c_int
+        L.c2t_lazy_step_gathered.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int32, P(c2t_accept_out),
+                                             C.c_void_p]
         L.c2t_expand_level_shard.restype = C.c_int
         L.c2t_expand_level_shard.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
                                              C.c_void_p]
@@ -397,6 +405,25 @@ class Context:
         assert t.shape[0] == self.B and t.shape[2] == self.V and t.stride(2) == 1
         _check(lib().c2t_accept_lazy(self._h, t.data_ptr(), t.stride(0), t.stride(1), C.byref(self._accept_c),
                                      _stream(stream)), "c2t_accept_lazy")
+
+    def c2t_lazy_begin(self, stream=None) -> None:
+        _check(lib().c2t_lazy_begin(self._h, C.byref(self._accept_c), _stream(stream)), "c2t_lazy_begin")
+
+    def c2t_lazy_argmax_shard(self, target_shard: torch.Tensor, vocab_begin: int, keys: torch.Tensor, stream=None) -> None:
+        """target_shard: [B, >=Nw, vocab_count] CUDA tensor of the configured dtype; keys: [B] int64 CUDA tensor."""
+        t = target_shard
+        assert t.is_cuda and t.dtype == self.cfg.torch_dtype and t.dim() == 3 and t.shape[0] == self.B
+        assert t.stride(2) == 1
+        assert keys.is_cuda and keys.dtype == torch.int64 and keys.is_contiguous() and keys.numel() == self.B
+        _check(lib().c2t_lazy_argmax_shard(self._h, t.data_ptr(), t.stride(0), t.stride(1), t.shape[2], vocab_begin,
+                                           keys.data_ptr(), _stream(stream)), "c2t_lazy_argmax_shard")
+
+    def c2t_lazy_step_gathered(self, round_: int, keys: torch.Tensor, stream=None) -> None:
+        """keys: [n_shards, B] int64 CUDA tensor of gathered keys."""
+        assert keys.is_cuda and keys.dtype == torch.int64 and keys.is_contiguous() and keys.dim() == 2
+        assert keys.shape[1] == self.B
+        _check(lib().c2t_lazy_step_gathered(self._h, round_, keys.data_ptr(), keys.shape[0], C.byref(self._accept_c),
+                                            _stream(stream)), "c2t_lazy_step_gathered")
 
     def c2t_status(self, stream=None):
         """(OR of all status words, per-sequence words as a list).  Synchronises the stream."""

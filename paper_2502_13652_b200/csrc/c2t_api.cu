@@ -481,13 +481,62 @@ int c2t_accept_lazy(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_str
   p.info = t.info_target;
   p.part_best = t.part_best;
   cudaStream_t s = (cudaStream_t)stream;
-  if (launch_lazy_walk_round(t, 0, out, s) != cudaSuccess) return C2T_ECUDA;
+  if (launch_lazy_walk_round(t, 0, out, nullptr, 0, s) != cudaSuccess) return C2T_ECUDA;
   ctx->launches += 1;
   for (int r = 0; r <= t.D; ++r) {   // a path has at most D + 1 nodes
     if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, s) != cudaSuccess) return C2T_ECUDA;
-    if (launch_lazy_walk_round(t, r + 1, out, s) != cudaSuccess) return C2T_ECUDA;
+    if (launch_lazy_walk_round(t, r + 1, out, nullptr, 0, s) != cudaSuccess) return C2T_ECUDA;
     ctx->launches += 2;
   }
+  return C2T_OK;
+}
+
+int c2t_lazy_begin(c2t_ctx *ctx, const c2t_accept_out *out, void *stream) {
+  if (!ctx) return C2T_EINVAL;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (launch_lazy_walk_round(ctx->t, 0, out, nullptr, 0, (cudaStream_t)stream) != cudaSuccess) return C2T_ECUDA;
+  ctx->launches += 1;
+  return C2T_OK;
+}
+
+int c2t_lazy_argmax_shard(c2t_ctx *ctx, const void *target_logits_dev, int64_t seq_stride, int64_t row_stride,
+                          int32_t vocab_count, int32_t vocab_begin, uint64_t *keys_dev, void *stream) {
+  if (!ctx || !target_logits_dev || !keys_dev) return C2T_EINVAL;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (vocab_count < 1 || vocab_begin < 0 || (int64_t)vocab_begin + vocab_count > ctx->cfg.vocab || seq_stride < 0 ||
+      row_stride < vocab_count)
+    return C2T_EINVAL;
+  if (!aligned16(target_logits_dev) || (seq_stride * ctx->elem_bytes) % 16 || (row_stride * ctx->elem_bytes) % 16)
+    return C2T_EALIGN;
+  const TreeState &t = ctx->t;
+  PassParams p;
+  memset(&p, 0, sizeof p);
+  p.logits = target_logits_dev; p.seq_stride = seq_stride; p.row_stride = row_stride;
+  p.V = vocab_count; p.K = 1; p.B = t.B; p.rows_per_seq_max = 1;
+  p.counts = t.walk_active;          // one row per sequence that is still walking ...
+  p.row_sel = t.walk_cur;            // ... the row of its current node
+  p.max_splits = t.max_splits_tgt;
+  p.n_slots = (int64_t)t.B * t.Nw * t.max_splits_tgt;
+  p.status = t.status;
+  p.info = t.info_target;
+  p.part_best = t.part_best;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (launch_argmax_pass(p, ctx->cfg.dtype, ctx->grid, s) != cudaSuccess) return C2T_ECUDA;
+  if (launch_export_lazy_best(t, vocab_begin, reinterpret_cast<unsigned long long *>(keys_dev), s) != cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 2;
+  return C2T_OK;
+}
+
+int c2t_lazy_step_gathered(c2t_ctx *ctx, int round, const uint64_t *keys_dev, int32_t n_shards,
+                           const c2t_accept_out *out, void *stream) {
+  if (!ctx || !keys_dev || n_shards < 1 || round < 1) return C2T_EINVAL;
+  if (n_shards > C2T_MAX_SHARDS) return C2T_ERANGE;
+  if (!ctx->finalized) return C2T_EORDER;
+  if (launch_lazy_walk_round(ctx->t, round, out, reinterpret_cast<const unsigned long long *>(keys_dev), n_shards,
+                             (cudaStream_t)stream) != cudaSuccess)
+    return C2T_ECUDA;
+  ctx->launches += 1;
   return C2T_OK;
 }
 

@@ -200,6 +200,9 @@ cudaError_t launch_accept_walk(const TreeState &t, const c2t_accept_out *out, co
                                int n_shards, cudaStream_t s);
 cudaError_t launch_export_best(const TreeState &t, int vocab_begin, unsigned long long *out, cudaStream_t s);
 // one round of the lazy walk: round 0 starts it, round r > 0 consumes the arg-max of round r-1
-cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s);
+// gathered == nullptr: the round consumes this context's own arg-max pass; else n_shards gathered keys per sequence
+cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out,
+                                   const unsigned long long *gathered, int n_shards, cudaStream_t s);
+cudaError_t launch_export_lazy_best(const TreeState &t, int vocab_begin, unsigned long long *out, cudaStream_t s);
 
 }  // namespace c2t

@@ -335,7 +335,10 @@ __global__ void __launch_bounds__(256) dense_mask_kernel(TreeState t, T *out, lo
 // all sequences, 1024 at a time; the scan numbers the walking sequences the way the pass did.
 constexpr int kWalkThreads = 1024;
 
-__global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState t, int round, c2t_accept_out out) {
+// gathered == nullptr: the arg-max of this context's own pass over whole rows; else the best of n_shards gathered keys
+// per sequence ([n_shards, B], one key for the sequence's current node, 0 for a sequence that has stopped).
+__global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState t, int round, c2t_accept_out out,
+                                                                       const unsigned long long *gathered, int n_shards) {
   __shared__ int s_warp[kWalkThreads / 32 + 1];
   chain_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -383,18 +386,25 @@ __global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState
     rows_before += s_warp[kWalkThreads / 32];
     if (!was) continue;
 
-    const long long first_vec = (long long)a * info.vec_per_row;
-    const int c_first = (int)(first_vec / info.span);
-    const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
-    int n_splits = c_last - c_first + 1;
-    if (n_splits > t.max_splits_tgt) {
-      n_splits = t.max_splits_tgt;
-      atomicOr(&t.status[b], C2T_ST_INTERNAL);
-    }
     unsigned long long best = 0ull;
-    for (int sp = 0; sp < n_splits; ++sp) {
-      const unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + sp];
-      best = k > best ? k : best;
+    if (gathered) {                                    // equal logits in two shards: the larger key is the lower token id
+      for (int sh = 0; sh < n_shards; ++sh) {
+        const unsigned long long k = gathered[(size_t)sh * t.B + b];
+        best = k > best ? k : best;
+      }
+    } else {
+      const long long first_vec = (long long)a * info.vec_per_row;
+      const int c_first = (int)(first_vec / info.span);
+      const int c_last = (int)((first_vec + info.vec_per_row - 1) / info.span);
+      int n_splits = c_last - c_first + 1;
+      if (n_splits > t.max_splits_tgt) {
+        n_splits = t.max_splits_tgt;
+        atomicOr(&t.status[b], C2T_ST_INTERNAL);
+      }
+      for (int sp = 0; sp < n_splits; ++sp) {
+        const unsigned long long k = t.part_best[(size_t)a * t.max_splits_tgt + sp];
+        best = k > best ? k : best;
+      }
     }
     const int want = best ? key_token(best) : -1;
     const int n = t.final_n[b];
@@ -417,6 +427,45 @@ __global__ void __launch_bounds__(kWalkThreads) lazy_walk_round_kernel(TreeState
   }
 }
 
+// After an arg-max pass over one token range of the walking sequences' current rows: per sequence the best key of
+// that range with the token id made global (0 for a sequence that has stopped), for c2t_lazy_argmax_shard.  The
+// pass numbered the walking sequences in sequence order; the scan here does the same.
+__global__ void __launch_bounds__(kWalkThreads) export_lazy_best_kernel(TreeState t, int tok_base, unsigned long long *out) {
+  __shared__ int s_warp[kWalkThreads / 32 + 1];
+  chain_enter();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const PassInfo info = *t.info_target;
+  int rows_before = 0;
+  for (int base = 0; base < t.B; base += kWalkThreads) {
+    const int b = base + tid;
+    const int was = b < t.B ? t.walk_active[b] : 0;
+    int inc = was;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += v;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (tid == 0) {
+      int run = 0;
+      for (int w = 0; w < kWalkThreads / 32; ++w) { const int v = s_warp[w]; s_warp[w] = run; run += v; }
+      s_warp[kWalkThreads / 32] = run;
+    }
+    __syncthreads();
+    const int a = rows_before + s_warp[warp] + inc - was;
+    rows_before += s_warp[kWalkThreads / 32];
+    if (b >= t.B) continue;
+    unsigned long long key = 0ull;
+    if (was) {
+      const unsigned long long best = row_best_key(t, info, b, a);
+      if (best) key = (best & 0xFFFFFFFF00000000ull) | (0xFFFFFFFFu - (uint32_t)(key_token(best) + tok_base));
+    }
+    out[b] = key;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_dense_mask(const TreeState &t, void *out, int out_dtype, int64_t kv_len, cudaStream_t s) {
@@ -431,11 +480,16 @@ cudaError_t launch_dense_mask(const TreeState &t, void *out, int out_dtype, int6
   return cudaGetLastError();
 }
 
-cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out, cudaStream_t s) {
+cudaError_t launch_lazy_walk_round(const TreeState &t, int round, const c2t_accept_out *out,
+                                   const unsigned long long *gathered, int n_shards, cudaStream_t s) {
   c2t_accept_out o;
   memset(&o, 0, sizeof o);
   if (out) o = *out;
-  return launch_chained(lazy_walk_round_kernel, dim3(1), dim3(kWalkThreads), 0, s, t, round, o);
+  return launch_chained(lazy_walk_round_kernel, dim3(1), dim3(kWalkThreads), 0, s, t, round, o, gathered, n_shards);
+}
+
+cudaError_t launch_export_lazy_best(const TreeState &t, int vocab_begin, unsigned long long *out, cudaStream_t s) {
+  return launch_chained(export_lazy_best_kernel, dim3(1), dim3(kWalkThreads), 0, s, t, vocab_begin, out);
 }
 
 cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,

@@ -55,6 +55,8 @@ class ExchangeBuffers:
         self.local = ctx.new_row_records(1)[0]                         # [B, F, bytes]
         self.keys = torch.zeros((world, ctx.B, ctx.Nw), dtype=torch.int64, device=self.records.device)
         self.local_keys = torch.zeros((ctx.B, ctx.Nw), dtype=torch.int64, device=self.records.device)
+        self.walk_keys = torch.zeros((world, ctx.B), dtype=torch.int64, device=self.records.device)
+        self.local_walk_keys = torch.zeros((ctx.B,), dtype=torch.int64, device=self.records.device)
 
 
 def vocab_parallel_level(ctx, level: int, shard_logits: torch.Tensor, vocab_begin: int,
@@ -78,3 +80,16 @@ def vocab_parallel_accept(ctx, target_shard: torch.Tensor, vocab_begin: int,
     buffers = buffers or ExchangeBuffers(ctx, group)
     ctx.c2t_argmax_shard(target_shard, vocab_begin, buffers.local_keys, stream)
     ctx.c2t_accept_gathered(gather_row_records(buffers.local_keys, group, buffers.keys), stream)
+
+
+
+def vocab_parallel_accept_lazy(ctx, target_shard: torch.Tensor, vocab_begin: int,
+                               group: Optional[dist.ProcessGroup] = None, stream=None,
+                               buffers: Optional[ExchangeBuffers] = None) -> None:
+    """The same walk reading only the target rows on the accepted path: D + 1 rounds of "this rank's best key of
+    every walking sequence's current row, an all-gather of 8 bytes per sequence, one step of every walk"."""
+    buffers = buffers or ExchangeBuffers(ctx, group)
+    ctx.c2t_lazy_begin(stream)
+    for r in range(1, ctx.D + 2):
+        ctx.c2t_lazy_argmax_shard(target_shard, vocab_begin, buffers.local_walk_keys, stream)
+        ctx.c2t_lazy_step_gathered(r, gather_row_records(buffers.local_walk_keys, group, buffers.walk_keys), stream)

@@ -331,6 +331,18 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
         for k in acc_g:
             assert np.array_equal(acc_s[k], acc_g[k]), f"sharded acceptance: {k} differs from the whole-row walk"
         assert np.array_equal(amax_s, view["node_argmax"])
+        # ... and the walk that reads only the rows it visits, sharded: D + 1 rounds of one key per sequence and range
+        lkeys = torch.zeros((len(shards), B), dtype=torch.int64, device=dev)
+        ctx.c2t_lazy_begin()
+        for r in range(1, D + 2):
+            for g, (v0, v1) in enumerate(shards):
+                ctx.c2t_lazy_argmax_shard(target_dev[:, :, v0:v1], v0, lkeys[g])
+            ctx.c2t_lazy_step_gathered(r, lkeys)
+        acc_ls = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+        amax_ls = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+        for k in acc_g:
+            assert np.array_equal(acc_ls[k], acc_g[k]), f"sharded lazy acceptance: {k} differs from the whole-row walk"
+        assert np.array_equal(amax_ls, amax_l), "sharded lazy acceptance read other rows than the whole-row lazy walk"
     ctx.c2t_accept(target_dev)                      # leave the all-rows results behind for the caller
     for b in seqs:
         tree, L, ft, ver, acc = orc[b]

@@ -479,12 +479,29 @@ def test_lazy_accept_follows_planted_paths():
     ctx.c2t_accept_lazy(tg); torch.cuda.synchronize()
     lazy = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
     amax_lazy = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
+    lazy = {k: v.copy() for k, v in lazy.items()}; amax_lazy = amax_lazy.copy()
+    # the same walk over target rows sharded into three token ranges (the planted tokens fall into different ranges)
+    shards = [(0, 2000), (2000, 6000), (6000, V)]
+    keys = torch.zeros((len(shards), B), dtype=torch.int64, device="cuda")
+    ctx.c2t_lazy_begin()
+    for r in range(1, D + 2):
+        for g, (v0, v1) in enumerate(shards):
+            ctx.c2t_lazy_argmax_shard(tg[:, :, v0:v1], v0, keys[g])
+        ctx.c2t_lazy_step_gathered(r, keys)
+    torch.cuda.synchronize()
+    lazy_s = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
+    amax_lazy_s = ctx.c2t_get_view()["node_argmax"].cpu().numpy()
     for b, chain in enumerate(planted):
-        assert full["accept_len"][b] == len(chain) - 1 == lazy["accept_len"][b]
+        assert full["accept_len"][b] == len(chain) - 1 == lazy["accept_len"][b] == lazy_s["accept_len"][b]
         assert [x for x in full["path"][b] if x >= 0] == chain == [x for x in lazy["path"][b] if x >= 0]
-        assert full["next_token"][b] == lazy["next_token"][b]
+        assert [x for x in lazy_s["path"][b] if x >= 0] == chain
+        assert full["next_token"][b] == lazy["next_token"][b] == lazy_s["next_token"][b]
         for i in range(Nw):
             assert amax_lazy[b, i] == (amax_full[b, i] if i in chain else -1)
+            assert amax_lazy_s[b, i] == amax_lazy[b, i]
+        # against the oracle: the arg-max of every row on the path, one by one
+        for i in chain:
+            assert amax_full[b, i] == oracle.row_argmax(target[b, i])
     assert max(len(c) for c in planted) >= 3
     ctx.close()
 
