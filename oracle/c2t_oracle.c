@@ -221,7 +221,7 @@ int orc_build_tree(const orc_config *cfg, const void *logits, int64_t level_stri
     const size_t esz = cfg->dtype == ORC_BF16 ? 2 : 4;
     int overflow = 0;
 
-    /* T <- {r}, C_r = 1, N <- {r} */
+    /* root initialisation (Alg. 1): the tree and the generator set hold the root alone, with confidence 1 */
     T->n = 1;
     T->tok[0] = root_tok; T->parent[0] = -1; T->level[0] = 0;
     T->logP[0] = 0.0; T->C[0] = 1.0; T->Chat[0] = INFINITY;
@@ -243,7 +243,7 @@ int orc_build_tree(const orc_config *cfg, const void *logits, int64_t level_stri
         double *cH = L->H + (size_t)d * FK, *cC = L->C + (size_t)d * FK;
         int32_t *ckeep = L->keep + (size_t)d * FK, *cnext = L->next + (size_t)d * FK;
 
-        /* N <- topK(M_d(N)): K most probable children of every generator */
+        /* children by generation probability (Sec. 4.2.2): the K most probable tokens of every generator's row */
         int32_t nc = 0;
         for (int32_t j = 0; j < nf; ++j) {
             const int32_t f = L->frontier_node[(size_t)d * F + j];
@@ -262,7 +262,7 @@ int orc_build_tree(const orc_config *cfg, const void *logits, int64_t level_stri
         }
         L->n_cand[d] = nc;
 
-        /* C_i <- F(P_i, H_i, d_i); remove i if C_i < beta */
+        /* confidence of every child (Eq. 4) and first pruning (Sec. 4.2.1): a child stays iff its confidence reaches beta */
         int32_t n_surv = 0;
         for (int32_t c = 0; c < nc; ++c) {
             double P = exp(clogP[c]);
@@ -282,7 +282,7 @@ int orc_build_tree(const orc_config *cfg, const void *logits, int64_t level_stri
         int32_t n_next = n_surv < F ? n_surv : F;
         for (int32_t s = 0; s < n_next; ++s) cnext[order[s].id] = 1;
 
-        /* extend N or topK(N) to T, in candidate order */
+        /* tree append (Alg. 1), in candidate order: the capped set, or every survivor (the variant of App. B.6) */
         int32_t slot = 0;
         for (int32_t c = 0; c < nc; ++c) {
             int add = cfg->tree_add == ORC_ADD_ALL_SURVIVORS ? ckeep[c] : cnext[c];
