@@ -45,9 +45,9 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  The counters
 # belong to the kernel sources whose hash stands beside them: when a source changes the hash no longer matches and
 # the bench reports no traffic figure until the counters (and the hash) are taken again.
-EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.09e6}
+EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.13e6}
 EXPAND_SOURCES = ("expand_pass.cu", "c2t_internal.h", "vocab_common.cuh")
-EXPAND_SOURCES_SHA16 = "d33adf80192b8868"
+EXPAND_SOURCES_SHA16 = "8c243392f679a8e7"
 
 
 def expand_dram_bytes():
@@ -72,7 +72,7 @@ def measured_hbm_peak():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled every 50 ms in a child process."""
+    """nvidia-smi clocks and throttle reasons, sampled every 20 ms in a child process."""
     FIELDS = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -82,7 +82,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
