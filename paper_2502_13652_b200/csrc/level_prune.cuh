@@ -257,6 +257,8 @@ struct PruneShared {
   float w[5 * C2T_MAX_HIDDEN + 4];
   float x[kMaxCand];
   int tok[kMaxCand];
+  double flogP[C2T_MAX_FRONTIER];              // joint log-probability of every frontier node
+  int fnode[C2T_MAX_FRONTIER];                 // tree id of every frontier node
   int rowfault[C2T_MAX_FRONTIER];
   int scan[NW + 1];
   int misc[2];
@@ -302,6 +304,14 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
   int n = t.frontier_n[cur][b];
   const int row_off = t.row_off_draft[b];         // rows of earlier sequences in the expand pass
   const PassInfo info = *t.info_draft;            // (loads issued together with the one above)
+  // the frontier's nodes and their joint log-probabilities (Eq. 1's left factor), fetched now so that their two
+  // dependent loads run beside the rows' merges (slots past the frontier's size hold anything: kept in bounds, unused)
+  if (tid < F) {
+    int f = t.frontier_node[cur][(size_t)b * F + tid];
+    f = f < 0 ? 0 : (f >= t.cap ? t.cap - 1 : f);
+    sh.fnode[tid] = f;
+    sh.flogP[tid] = t.tree_logP[(size_t)b * t.cap + f];
+  }
   n = n < 0 ? 0 : (n > F ? F : n);
   const size_t cbase = (size_t)b * F * K;
 
@@ -342,12 +352,11 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
   const int nc = n * K;
   for (int c = tid; c < nc; c += kTreeThreads) {
     const int j = c / K;
-    const int f = t.frontier_node[cur][(size_t)b * F + j];
     const int tok = s_tok[c];
     const float x = s_x[c];
     const bool ok = tok >= 0 && !s_rowfault[j];
     const double lp = (x > kNegInfAsFinite) ? ((double)x - s_rowM[j]) - s_rowL[j] : -INFINITY;
-    const double logP = t.tree_logP[(size_t)b * t.cap + f] + lp;           // Eq. 1 in log space
+    const double logP = sh.flogP[j] + lp;                                   // Eq. 1 in log space
     const double P = exp(logP);
     const double H = s_rowH[j];
     double C;
@@ -413,7 +422,7 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
     const int id = base + off_add++;
     if (id < t.cap) {
       const int j = c / K;
-      const int f = t.frontier_node[cur][(size_t)b * F + j];
+      const int f = sh.fnode[j];
       t.tree_token[tb + id] = s_tok[c];
       t.tree_parent[tb + id] = f;
       t.tree_level[tb + id] = level + 1;

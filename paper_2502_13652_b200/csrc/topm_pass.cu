@@ -20,9 +20,13 @@
 namespace c2t {
 namespace {
 
-constexpr int kTopmThreads = 1024;
+#ifndef C2T_TOPM_THREADS
+#define C2T_TOPM_THREADS 1024
+#define C2T_TOPM_CAND 32768
+#endif
+constexpr int kTopmThreads = C2T_TOPM_THREADS;
 constexpr int kTopmBatch = 8;          // independent 16-byte loads a thread keeps in flight
-constexpr int kTopmCand = 32768;       // candidate keys the fast path can hold in shared memory (128 KB)
+constexpr int kTopmCand = C2T_TOPM_CAND;   // candidate keys the fast path can hold in shared memory
 
 // Where the expand pass, which runs just before, left what this pass can reuse: the row's maximum
 // is the largest of the keys held out of its partial sums.
@@ -241,6 +245,47 @@ __global__ void __launch_bounds__(kTopmThreads) topm_entropy_kernel(const void *
   // bins are visited four at a time from there downwards and the bulk of the row is never counted.
   if (!all) {
     int d0 = (int)(f32_orderable(__float_as_uint(m)) >> 24);
+    // The M-th largest can lie far below the maximum's bin (a positive maximum and a negative M-th largest are half
+    // the key space apart): one sweep over the top four key bits first, so that the fine count starts at most
+    // sixteen bins above its goal.
+    if (tid < 16) s_hist[tid] = 0u;
+    __syncthreads();
+    for (int it0 = 0; it0 < sweeps; it0 += kTopmBatch) {
+      uint4 qb[kTopmBatch];
+#pragma unroll
+      for (int k = 0; k < kTopmBatch; ++k) {
+        const int vec = (it0 + k) * kTopmThreads + tid;
+        qb[k] = vec < vpr ? VT::load(row, vec, v_full, V) : make_uint4(lo, lo, lo, lo);
+      }
+#pragma unroll
+      for (int k = 0; k < kTopmBatch; ++k) {
+        const int vec = (it0 + k) * kTopmThreads + tid;
+        float x[VT::N];
+        VT::clamp(qb[k]);
+        VT::unpack(qb[k], x);
+#pragma unroll
+        for (int i = 0; i < VT::N; ++i) {
+          unsigned bin = 0xFFFFFFFFu;
+          if (vec < vpr && vec * VT::N + i < V && x[i] == x[i]) bin = f32_orderable(__float_as_uint(x[i])) >> 28;
+          const unsigned peers = __match_any_sync(kFull, bin);
+          if (bin != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (unsigned)__popc(peers));
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned need = s_need;
+      int cb = 15;
+      for (; cb > 0 && s_hist[cb] < need; --cb) need -= s_hist[cb];
+      s_need = need;                               // still wanted from coarse bin cb downwards
+      s_found = cb;
+    }
+    __syncthreads();
+    {
+      const int top_of_coarse = s_found * 16 + 15;
+      d0 = d0 < top_of_coarse ? d0 : top_of_coarse;
+    }
+    __syncthreads();
     for (;;) {
       unsigned c[4] = {0u, 0u, 0u, 0u};
       if (tid < 4) s_win[tid] = 0u;
