@@ -115,6 +115,14 @@ def _vp_worker(rank: int, world: int, port: int, out):
     v0, v1 = vp.shard_ranges(V, world, 4)[rank]
     local = torch.from_numpy(_range_records(logits, v0, v1, K).view(np.uint8).reshape(B, F, RECORD.itemsize))
     gathered = vp.gather_row_records(local)                           # the path's only collective
+    # the same exchange into a buffer allocated once (what ExchangeBuffers holds), and for the 8-byte keys of the
+    # acceptance walks: [B, Nw] per rank for the all-rows walk, [B] per rank and round for the lazy one
+    buf = torch.full((world, B, F, RECORD.itemsize), 255, dtype=torch.uint8)
+    again = vp.gather_row_records(local, out=buf)
+    assert again.data_ptr() == buf.data_ptr() and torch.equal(again, gathered)
+    keys = torch.arange(B, dtype=torch.int64) * 10 + rank
+    got_keys = vp.gather_row_records(keys, out=torch.zeros((world, B), dtype=torch.int64))
+    assert got_keys.tolist() == [[b * 10 + r for b in range(B)] for r in range(world)]
     if rank == 0:
         out.put(gathered.numpy())
     dist.barrier()
