@@ -83,7 +83,9 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   const size_t B = c->batch, F = c->frontier_cap, K = c->topk;
   const size_t cap = tree_capacity_unchecked(c), Nw = c2t_final_width(c);
   const int eb = c->dtype == C2T_BF16 ? 2 : 4;
-  const size_t ms = max_splits_for(c->vocab, eb, kMaxSms * kExpandCtasPerSm * kExpandWarps, kSegmentPad);   // expand workers outnumber arg-max CTAs
+  // (expand workers outnumber arg-max CTAs, and their spans may be shorter)
+  const size_t ms = max_splits_for(c->vocab, eb, kMaxSms * kExpandCtasPerSm * kExpandWarps, kSegmentPad,
+                                   expand_min_span(c->vocab, eb, c->topk));
   TreeState s;
   memset(&s, 0, sizeof s);
   for (int i = 0; i < 2; ++i) {
@@ -179,7 +181,8 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   if (workspace_bytes < carve(cfg, nullptr, nullptr)) return C2T_ERANGE;
   if (cudaSetDevice(cfg->device) != cudaSuccess) { cudaGetLastError(); return C2T_ECUDA; }
   const int grid = pass_grid(cfg->device);
-  if (grid < 0 || prepare_expand_pass() != cudaSuccess || prepare_topm_pass() != cudaSuccess) {
+  if (grid < 0 || prepare_expand_pass() != cudaSuccess || prepare_topm_pass() != cudaSuccess ||
+      prepare_tree_kernels() != cudaSuccess) {
     cudaGetLastError();
     return C2T_ECUDA;
   }
@@ -200,7 +203,8 @@ int c2t_init(const c2t_config *cfg, void *workspace_dev, size_t workspace_bytes,
   t.hidden = cfg->classifier == C2T_CLS_MLP ? cfg->hidden : 0;
   t.classifier = cfg->classifier; t.tree_add = cfg->tree_add; t.beta = cfg->threshold;
   t.entropy_top_m = cfg->entropy_top_m;
-  t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid_expand * kExpandWarps, kSegmentPad);
+  t.min_span = expand_min_span(cfg->vocab, (int)ctx->elem_bytes, cfg->topk);
+  t.max_splits = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid_expand * kExpandWarps, kSegmentPad, t.min_span);
   t.max_splits_tgt = max_splits_for(cfg->vocab, (int)ctx->elem_bytes, ctx->grid, 0);
 
   cudaError_t e = cudaSuccess;
@@ -249,6 +253,7 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   p.V = t.V; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
   p.counts = t.frontier_n[level & 1];
   p.max_splits = t.max_splits;
+  p.min_span = t.min_span;
   p.n_slots = (int64_t)t.B * t.F * t.max_splits;
   p.status = t.status;
   p.info = t.info_draft;
@@ -305,6 +310,7 @@ int c2t_expand_prune_level(c2t_ctx *ctx, int level, const void *logits_dev, int6
   p.V = t.V; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
   p.counts = t.frontier_n[level & 1];
   p.max_splits = t.max_splits;
+  p.min_span = t.min_span;
   p.n_slots = (int64_t)t.B * t.F * t.max_splits;
   p.status = t.status;
   p.info = t.info_draft;
@@ -334,6 +340,7 @@ int c2t_expand_level_shard(c2t_ctx *ctx, int level, const void *logits_dev, int6
   p.V = vocab_count; p.K = t.K; p.B = t.B; p.rows_per_seq_max = t.F;
   p.counts = t.frontier_n[level & 1];
   p.max_splits = t.max_splits;                    // sized for whole rows: enough for any part of one
+  p.min_span = t.min_span;
   p.n_slots = (int64_t)t.B * t.F * t.max_splits;
   p.status = t.status;
   p.info = t.info_draft;

@@ -121,6 +121,7 @@ struct PassParams {
   const int32_t *counts;            // [B] active rows per sequence, device
   const int32_t *row_sel;           // arg-max pass only, may be null: [B] the row of sequence b to read (then counts is 0 or 1)
   int32_t max_splits;               // partial slots per row
+  int32_t min_span;                 // expand: the fewest vectors a worker gets (expand_min_span)
   int64_t n_slots;                  // partial slots in the workspace (rows the workspace was carved for x max_splits)
   uint32_t *status;                 // may be null: a status word for C2T_ST_INTERNAL (the first sequence's)
   PassInfo *info;                   // written by CTA 0
@@ -134,7 +135,12 @@ struct PassParams {
 };
 
 // partial slots a row can need; workers: CTAs (arg-max, pad 0) or warps (expand, pad kSegmentPad)
-int max_splits_for(int vocab, int elem_bytes, int workers, int pad);
+int max_splits_for(int vocab, int elem_bytes, int workers, int pad, int min_span = kMinSpanVectors);
+// Keys of a row's partial lists that one warp of the row merge stages in shared memory; a row with more takes a slow path.
+constexpr int kStageKeys = 320;
+// The fewest vectors a worker of the expand pass gets: as few as the row merge allows (at most 31 partial lists per
+// row, and K keys apiece must fit the staging area), so that launches with few rows still spread over the chip.
+int expand_min_span(int vocab, int elem_bytes, int K);
 
 cudaError_t prepare_expand_pass();   // once per device: opt in to the kernel's shared-memory size
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s);
@@ -146,7 +152,7 @@ cudaError_t launch_expand_prune(const PassParams &p, const TreeState &t, int lev
 // ---------------------------------------------------------------- tree state -
 
 struct TreeState {
-  int32_t B, V, K, F, D, N, Nw, W, cap, hidden, classifier, tree_add, max_splits, max_splits_tgt;
+  int32_t B, V, K, F, D, N, Nw, W, cap, hidden, classifier, tree_add, max_splits, max_splits_tgt, min_span;
   float beta;
   // frontier, double buffered by level parity
   int32_t *frontier_n[2];      // [B]
@@ -182,6 +188,7 @@ struct TreeState {
 // truncated entropy (Eq. 3): per active row (b, j) the sums over its M largest logits, out[b * F + j] = {S_M, T_M};
 // runs after the expand pass of the same level, whose partial records give it the row maxima
 cudaError_t prepare_topm_pass();     // once per device: opt in to the kernel's shared-memory size
+cudaError_t prepare_tree_kernels();  // the same for the pruning kernel
 cudaError_t launch_topm_entropy(const void *logits, int64_t seq_stride, int64_t row_stride, int V, int M, int F,
                                 int B, const int32_t *counts, const TreeState &t, double2 *out, int dtype,
                                 cudaStream_t s);

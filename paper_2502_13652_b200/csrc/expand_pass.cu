@@ -456,7 +456,7 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
   const long long vtotal = (long long)n_rows * vrow;
   const long long workers = (long long)gridDim.x * kEWarps;
   long long span = div_floor(vtotal + workers - 1, workers);
-  if (span < kMinSpanVectors) span = kMinSpanVectors;
+  if (span < p.min_span) span = p.min_span;
   // consecutive workers sit on different SMs: a launch with few rows (level 0) still uses every SM
   const long long worker = (long long)warp * gridDim.x + blockIdx.x;
   if (worker == 0 && lane == 0) {
@@ -603,10 +603,19 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_prune
 
 }  // namespace
 
-int max_splits_for(int vocab, int elem_bytes, int workers, int pad) {
+int expand_min_span(int vocab, int elem_bytes, int K) {
   const int vec = 16 / elem_bytes;
   const int vec_per_row = (vocab + vec - 1) / vec;
-  int by_span = (vec_per_row + pad + kMinSpanVectors - 1) / kMinSpanVectors;
+  int lists = kStageKeys / (K < 1 ? 1 : K) - 1;      // one list in reserve: a row's pieces may start mid-worker
+  lists = lists > 31 ? 31 : (lists < 4 ? 4 : lists);
+  const int span = (vec_per_row + kSegmentPad + lists - 1) / lists;
+  return span < 256 ? 256 : span;
+}
+
+int max_splits_for(int vocab, int elem_bytes, int workers, int pad, int min_span) {
+  const int vec = 16 / elem_bytes;
+  const int vec_per_row = (vocab + vec - 1) / vec;
+  int by_span = (vec_per_row + pad + min_span - 1) / min_span;
   if (by_span > workers) by_span = workers;
   return by_span + 1;
 }

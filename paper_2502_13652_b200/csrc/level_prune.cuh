@@ -9,7 +9,6 @@ namespace c2t {
 namespace {
 
 constexpr int kMaxCand = C2T_MAX_TOPK * C2T_MAX_FRONTIER;   // 1024
-constexpr int kStageKeys = 192;   // keys of a row's partial lists that a warp stages in shared memory
 constexpr unsigned kFullMask = 0xFFFFFFFFu;
 
 __device__ __forceinline__ double warp_sum(double v) {

@@ -59,7 +59,8 @@ __global__ void __launch_bounds__(kTreeThreads) export_rows_kernel(TreeState t, 
 // records == nullptr: the rows come from this context's own expand pass; else from gathered records of n_shards shards
 __global__ void __launch_bounds__(kTreeThreads) prune_level_kernel(TreeState t, int level, c2t_frontier out,
                                                                    const c2t_row_record *records, int n_shards) {
-  __shared__ PruneShared<kTreeWarps> sh;
+  extern __shared__ __align__(16) unsigned char s_prune[];
+  PruneShared<kTreeWarps> &sh = *reinterpret_cast<PruneShared<kTreeWarps> *>(s_prune);
   prune_level_body<kTreeThreads, true>(t, level, out, records, n_shards, blockIdx.x, sh);
 }
 
@@ -506,7 +507,13 @@ cudaError_t launch_prune_level(const TreeState &t, int level, const c2t_frontier
                                int n_shards, cudaStream_t s) {
   c2t_frontier o = {nullptr, nullptr, nullptr, nullptr};
   if (out) o = *out;
-  return launch_chained(prune_level_kernel, dim3(t.B), dim3(kTreeThreads), 0, s, t, level, o, records, n_shards);
+  return launch_chained(prune_level_kernel, dim3(t.B), dim3(kTreeThreads), sizeof(PruneShared<kTreeWarps>), s, t, level, o,
+                        records, n_shards);
+}
+
+cudaError_t prepare_tree_kernels() {
+  return cudaFuncSetAttribute(prune_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)sizeof(PruneShared<kTreeWarps>));
 }
 
 cudaError_t launch_final_prune(const TreeState &t, cudaStream_t s) {
