@@ -97,7 +97,7 @@ typedef struct {
   float   threshold;      /* beta; a node is kept iff C >= beta                           */
   int32_t entropy_top_m;  /* M of Eq. 3: entropy over the M most probable tokens, their
                              probabilities not renormalised; 0 (or M >= V) = exact, Eq. 2.
-                             M > 0 costs one more pass over the draft logits per level      */
+                             M > 0 adds a pool of a third of [B, F, V] to the workspace     */
   int32_t classifier;     /* c2t_classifier                                               */
   int32_t hidden;         /* h                                                            */
   const float *w1;        /* HOST [h*3] row-major, features in the order (P, H, d)        */
@@ -135,8 +135,10 @@ int c2t_begin_step(c2t_ctx *ctx, const int32_t *root_tok_dev, const int32_t *pre
  * for every active frontier slot (b, j), j < n_level(b), one pass over logits row (b, j)
  * yields the softmax normaliser, the exact entropy of the row and its K most probable
  * tokens (ties to the lower token id).  Results stay in the workspace for c2t_prune.
- * With cfg.entropy_top_m = M, 0 < M < V, a second kernel reads the active rows once more for
- * the entropy over the M most probable tokens (Eq. 3) that c2t_prune then uses instead.
+ * With cfg.entropy_top_m = M, 0 < M < V, the pass also sets aside the vectors that can hold one
+ * of a row's M most probable tokens, and a second kernel takes the entropy over those M (Eq. 3),
+ * which c2t_prune then uses instead, from them; only a row for which they do not suffice (see
+ * c2t_view.topm_from_pass) is read once more.
  *   logits_dev: [B, F, V] of cfg.dtype; element offset of (b, j, v) =
  *               b*seq_stride + j*row_stride + v.  Base address 16-byte aligned, both strides
  *               multiples of 16 bytes.  Rows of inactive slots are never read.
@@ -404,6 +406,9 @@ typedef struct {
   const int32_t *final_src;     /* [B, Nw] tree id each final node came from               */
   const int32_t *final_token, *final_parent, *final_level;
   const int32_t *node_argmax;   /* [B, Nw] target argmax per final node (after c2t_accept) */
+  const int32_t *topm_from_pass;/* [B, F] with 0 < entropy_top_m < V, else NULL: 1 where the last
+                                   c2t_expand_level took the row's Eq. 3 sums from the vectors the
+                                   pass set aside, 0 where the row was read a second time   */
 } c2t_view;
 int c2t_get_view(c2t_ctx *ctx, c2t_view *out);
 

@@ -69,7 +69,7 @@ class c2t_accept_out(C.Structure):
 _VIEW_FIELDS = ("tree_n", "tree_token", "tree_parent", "tree_level", "tree_logP", "tree_C", "tree_Chat",
                 "cand_n", "cand_token", "cand_lp", "cand_logP", "cand_H", "cand_C", "cand_flags",
                 "frontier_n", "frontier_node", "final_n", "final_src", "final_token", "final_parent",
-                "final_level", "node_argmax")
+                "final_level", "node_argmax", "topm_from_pass")
 
 
 class c2t_view(C.Structure):
@@ -441,11 +441,14 @@ class Context:
         _check(lib().c2t_get_view(self._h, C.byref(v)), "c2t_get_view")
         B, F, K, cap, Nw = self.B, self.F, self.K, self.cap, self.Nw
         shapes = {"tree_n": (B,), "cand_n": (B,), "frontier_n": (B,), "final_n": (B,),
-                  "frontier_node": (B, F)}
+                  "frontier_node": (B, F), "topm_from_pass": (B, F)}
         out = {}
         base = self.workspace.data_ptr()
         for name in _VIEW_FIELDS:
             ptr = getattr(v, name)
+            if not ptr:                      # (topm_from_pass without a truncated entropy)
+                out[name] = None
+                continue
             if name in shapes:
                 shape = shapes[name]
             elif name.startswith("tree_"):

@@ -124,6 +124,12 @@ size_t carve(const c2t_config *c, void *base, TreeState *t) {
   s.info_target = w.take<PassInfo>(1);
   s.row_off_draft = w.take<int32_t>(B + 1);
   s.topm = w.take<double2>(B * F);
+  if (c->entropy_top_m > 0 && c->entropy_top_m < c->vocab) {   // the expand pass sets Eq. 3's candidates aside
+    s.topm_pool_vecs = (long long)topm_pool_vectors(B, F, c->vocab, eb);
+    s.topm_pool = w.take<uint4>((size_t)s.topm_pool_vecs);
+    s.topm_seg = w.take<TopmSegment>(B * F * ms);
+    s.topm_done = w.take<int32_t>(B * F);
+  }
   s.part_stats = w.take<float4>(B * F * ms);
   s.part_keys = w.take<unsigned long long>(B * F * ms * K);
   s.part_held = w.take<unsigned long long>(B * F * ms * kHeldPerSlot);
@@ -259,14 +265,19 @@ int c2t_expand_level(c2t_ctx *ctx, int level, const void *logits_dev, int64_t se
   p.info = t.info_draft;
   p.part_stats = t.part_stats; p.part_keys = t.part_keys; p.part_held = t.part_held;
   p.row_off = t.row_off_draft;
+  const bool truncated = t.entropy_top_m > 0 && t.entropy_top_m < t.V;   // Eq. 3: the sums over the M most probable tokens
+  if (truncated) { p.topm_pool = t.topm_pool; p.topm_pool_vecs = t.topm_pool_vecs; p.topm_seg = t.topm_seg; }
   if (launch_expand_pass(p, ctx->cfg.dtype, ctx->grid_expand, (cudaStream_t)stream) != cudaSuccess)
     return C2T_ECUDA;
   ctx->launches += 1;
-  if (t.entropy_top_m > 0 && t.entropy_top_m < t.V) {   // Eq. 3: the sums over the M most probable tokens
-    if (launch_topm_entropy(logits_dev, seq_stride, row_stride, t.V, t.entropy_top_m, t.F, t.B, p.counts, t, t.topm,
-                            ctx->cfg.dtype, (cudaStream_t)stream) != cudaSuccess)
+  if (truncated) {
+    // from the vectors the pass set aside; then, for the rows where those did not suffice, from the rows themselves
+    if (launch_topm_finish(t.entropy_top_m, t.F, t.B, p.counts, t, t.topm, ctx->cfg.dtype, (cudaStream_t)stream) != cudaSuccess)
       return C2T_ECUDA;
-    ctx->launches += 1;
+    if (launch_topm_entropy(logits_dev, seq_stride, row_stride, t.V, t.entropy_top_m, t.F, t.B, p.counts, t, t.topm,
+                            t.topm_done, ctx->grid_expand, ctx->cfg.dtype, (cudaStream_t)stream) != cudaSuccess)
+      return C2T_ECUDA;
+    ctx->launches += 2;
   }
   ctx->expanded = 1;
   return C2T_OK;
@@ -575,6 +586,7 @@ int c2t_get_view(c2t_ctx *ctx, c2t_view *v) {
   v->frontier_node = t.frontier_node[ctx->next_level & 1];
   v->final_n = t.final_n; v->final_src = t.final_src; v->final_token = t.final_token;
   v->final_parent = t.final_parent; v->final_level = t.final_level; v->node_argmax = t.node_argmax;
+  v->topm_from_pass = t.topm_done;
   return C2T_OK;
 }
 

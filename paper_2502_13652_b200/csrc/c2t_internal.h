@@ -113,6 +113,8 @@ struct PassInfo {
   int32_t reserved;
 };
 
+struct TopmSegment;
+
 struct PassParams {
   const void *logits;
   int64_t seq_stride, row_stride;   // elements
@@ -130,9 +132,33 @@ struct PassParams {
   float4 *part_stats;               // {offset c, S, U, n_keys as int bits}: base-2 sums, see expand_pass.cu
   unsigned long long *part_keys;    // [.. * K] the segment's K largest keys, sorted descending, 0-padded
   unsigned long long *part_held;    // [.. * kHeldPerSlot] keys excluded from S and U (0 = none)
+  // expand with M > 0 (else null): the pool of candidate vectors, cut evenly among the workers, and a record per (row, split)
+  uint4 *topm_pool;
+  long long topm_pool_vecs;
+  TopmSegment *topm_seg;
   // argmax: per (row, split) best key
   unsigned long long *part_best;
 };
+
+// ---------------------------------------------------------------- candidates of the truncated entropy (Eq. 3)
+// With entropy_top_m = M > 0 the expand pass also sets aside every 16-byte vector that holds an element at or above
+// a floor of its segment: the kTopmRank-th largest of the 32 lane maxima over the segment's first two groups, about
+// the top 2 % of the elements seen there (M = 1000 of 128256 is the top 0.8 %).  The vectors go, in stream order, to
+// a region of the warp's own in a pool in global memory; the segment's record says where they are and what the floor
+// was.  A small kernel per row then takes the elements at or above the row's highest floor F from those vectors: if
+// there are at least M of them the M-th largest is among them and so is everything above it, and Eq. 3's sums follow
+// without reading the row again.  Rows for which that fails (a region ran full, fewer than M elements at or above F,
+// more than fit in shared memory) are left to the pass that reads the row again.
+constexpr int kTopmRank = 24;
+constexpr int kTopmPoolDivisor = 3;      // the pool holds a third of the largest level's vectors (twice what is expected)
+constexpr float kTopmLowestFloor = -1.7e38f;   // above -2^127, the value that pads a ragged vector
+struct TopmSegment {
+  int first;       // the segment's first vector in the pool
+  int n;           // vectors, or -1: the region ran full
+  float floor;
+  int pad;
+};
+size_t topm_pool_vectors(size_t batch, size_t rows_per_seq, int vocab, int elem_bytes);
 
 // partial slots a row can need; workers: CTAs (arg-max, pad 0) or warps (expand, pad kSegmentPad)
 int max_splits_for(int vocab, int elem_bytes, int workers, int pad, int min_span = kMinSpanVectors);
@@ -174,6 +200,10 @@ struct TreeState {
   int32_t *walk_active, *walk_cur, *walk_len;       // [B] state of the lazy acceptance walk
   int32_t entropy_top_m;       // M of Eq. 3 (0: exact entropy)
   double2 *topm;               // [B, F] {S_M, T_M} of the last expand call when M > 0
+  uint4 *topm_pool;            // M > 0: candidate vectors set aside by the expand pass
+  long long topm_pool_vecs;
+  TopmSegment *topm_seg;       // M > 0: [B * F * max_splits] where each segment's candidates are
+  int32_t *topm_done;          // M > 0: [B, F] 1 where the row's sums came from the candidate vectors
   uint32_t *status;            // [B]
   uint32_t *ticket;            // one counter: CTAs of a fused expand + prune launch that have finished (0 between launches)
   PassInfo *info_draft, *info_target;
@@ -190,8 +220,12 @@ struct TreeState {
 cudaError_t prepare_topm_pass();     // once per device: opt in to the kernel's shared-memory size
 cudaError_t prepare_tree_kernels();  // the same for the pruning kernel
 cudaError_t launch_topm_entropy(const void *logits, int64_t seq_stride, int64_t row_stride, int V, int M, int F,
-                                int B, const int32_t *counts, const TreeState &t, double2 *out, int dtype,
-                                cudaStream_t s);
+                                int B, const int32_t *counts, const TreeState &t, double2 *out, const int32_t *done,
+                                int n_ctas, int dtype, cudaStream_t s);
+// the same sums from the candidate vectors of the expand pass, for the rows where they suffice (t.topm_done says
+// which; launch_topm_entropy skips those when given t.topm_done)
+cudaError_t launch_topm_finish(int M, int F, int B, const int32_t *counts, const TreeState &t, double2 *out, int dtype,
+                               cudaStream_t s);
 cudaError_t launch_begin_step(const TreeState &t, const int32_t *root_tok, const int32_t *prefix_len,
                               cudaStream_t s);
 // records == nullptr: rows merged from this context's own expand pass; else from n_shards gathered records per row

@@ -256,9 +256,10 @@ __device__ __forceinline__ float value_just_above(uint32_t orderable) {
 }
 
 // The filter and the reference of a new segment, from the lane maxima over its first two
-// groups (the first is in registers, the second has just landed in the ring).
-template <bool BF16>
-__device__ __noinline__ float2 segment_warmup(int K, Group g, int vt, int v1, int v_full, const uint4 *next_slot) {
+// groups (the first is in registers, the second has just landed in the ring); TOPM: also the
+// floor of the candidate collection (.z).
+template <bool BF16, bool TOPM>
+__device__ __noinline__ float4 segment_warmup(int K, Group g, int vt, int v1, int v_full, const uint4 *next_slot) {
   using VT = Vec<BF16>;
   const int lane = threadIdx.x & 31;
   float lmax = -INFINITY;
@@ -280,17 +281,22 @@ __device__ __noinline__ float2 segment_warmup(int K, Group g, int vt, int v1, in
       if (vm == vm) lmax = fmaxf(lmax, vm);
     }
   }
-  uint32_t live = f32_orderable(__float_as_uint(lmax)), kth = 0, first = 0;
-  for (int r = 0; r < K; ++r) {            // K-th largest lane maximum
-    kth = __reduce_max_sync(kFull, live);
-    if (r == 0) first = kth;
-    const unsigned bal = __ballot_sync(kFull, live == kth);
+  uint32_t live = f32_orderable(__float_as_uint(lmax)), kth = 0, first = 0, low = 0;
+  const int rounds = TOPM && K < kTopmRank ? kTopmRank : K;
+  for (int r = 0; r < rounds; ++r) {       // K-th largest lane maximum
+    const uint32_t cur = __reduce_max_sync(kFull, live);
+    if (r == 0) first = cur;
+    if (r == K - 1) kth = cur;
+    if (TOPM && r == kTopmRank - 1) low = cur;
+    const unsigned bal = __ballot_sync(kFull, live == cur);
     if (lane == __ffs(bal) - 1) live = 0;
   }
   const uint32_t none = f32_orderable(0xFF800000u);   // -inf: a lane without data
-  float2 out;
+  float4 out;
   out.x = kth <= none ? -INFINITY : __uint_as_float(f32_from_orderable(kth));      // filter
   out.y = first <= none ? 0.f : __uint_as_float(f32_from_orderable(first));        // reference (any finite value if no data)
+  out.z = low <= none ? kTopmLowestFloor : fmaxf(__uint_as_float(f32_from_orderable(low)), kTopmLowestFloor);
+  out.w = 0.f;
   return out;
 }
 
@@ -384,15 +390,33 @@ __device__ __forceinline__ Drained drain_queue(WarpShared *ws, int qn, int K, Ac
   return d;
 }
 
+// Candidates of the truncated entropy (Eq. 3): where a warp puts the vectors whose largest element reaches its
+// segment's floor (ballot-ranked places in stream order, so the result does not depend on timing).
+struct TopmState {
+  uint4 *region;              // the warp's part of the pool
+  int cap, n, first;          // its size in vectors; vectors set aside by the warp so far (may pass cap: then nothing more is stored); n when the segment began
+  float floor;
+};
+
 // One group: vectors that meet the filter go to the queue, the others into the sums.  WHOLE:
-// no lane is past the segment's end.
-template <bool BF16, bool WHOLE>
-__device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, SegState &st, int vt, int v1,
+// no lane is past the segment's end (a vector past it holds the lowest value, below every floor).
+template <bool BF16, bool WHOLE, bool TOPM>
+__device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, SegState &st, TopmState &ts, int vt, int v1,
                                               unsigned lt_mask, uint32_t *status) {
   using VT = Vec<BF16>;
   float vm[kVPL];
 #pragma unroll
   for (int u = 0; u < kVPL; ++u) vm[u] = VT::vmax(g.q[u]);
+  if (TOPM) {
+#pragma unroll
+    for (int u = 0; u < kVPL; ++u) {
+      const bool c = vm[u] >= ts.floor;              // (false for a vector with a NaN; such a row is reported anyway)
+      const unsigned cm = __ballot_sync(kFull, c);
+      const int pos = ts.n + __popc(cm & lt_mask);
+      if (c && pos < ts.cap) ts.region[pos] = g.q[u];
+      ts.n += __popc(cm);
+    }
+  }
   float gm = vm[0];
 #pragma unroll
   for (int u = 1; u < kVPL; ++u) gm = fmaxf(gm, vm[u]);
@@ -439,7 +463,7 @@ __device__ __forceinline__ void drain_into(WarpShared *ws, SegState &st, int K, 
 // ---------------------------------------------------------------- the kernel
 
 // The pass itself: what every warp of the grid does (a warp returns when its span is done).
-template <bool BF16>
+template <bool BF16, bool TOPM>
 __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned char *s_dyn) {
   using VT = Vec<BF16>;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -487,11 +511,20 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
 
   const unsigned lt_mask = (1u << lane) - 1u;
   SegState st;
+  TopmState ts;
+  ts.region = nullptr; ts.cap = 0; ts.n = 0; ts.first = 0; ts.floor = INFINITY;
+  if (TOPM) {
+    const long long busy = div_floor(vtotal + span - 1, span);       // workers with a span of this launch
+    const long long cap = div_floor(p.topm_pool_vecs, busy > 0 ? busy : 1);
+    ts.cap = (int)(cap < 0x3FFFFFFF ? cap : 0x3FFFFFFF);
+    ts.region = p.topm_pool + worker * ts.cap;
+  }
   bool fresh = true;                                 // the current group opens a segment
   for (;;) {
     const Segment seg = cur.seg;
     if (fresh) {
-      const float2 w = segment_warmup<BF16>(K, g, cur.tv0 + lane, seg.v1, v_full, ws->ring[next_slot(n)]);
+      const float4 w = segment_warmup<BF16, TOPM>(K, g, cur.tv0 + lane, seg.v1, v_full, ws->ring[next_slot(n)]);
+      if (TOPM) { ts.floor = w.z; ts.first = ts.n; }
       st.acc.S0 = st.acc.S1 = st.acc.U0 = st.acc.U1 = 0.f;
       st.thr = w.x;
       st.m = w.y;
@@ -509,7 +542,7 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
         const uint4 *src = reinterpret_cast<const uint4 *>(seg.row) + pre.tv0 + lane;
         int vt = cur.tv0 + lane;
         for (int i = 0; i < k; ++i) {
-          process_group<BF16, true>(ws, g, st, vt, 0, lt_mask, p.status);
+          process_group<BF16, true, TOPM>(ws, g, st, ts, vt, 0, lt_mask, p.status);
           n = next_slot(n);
           vt += kGroupVecs;
           cp_async_wait<kRingSlots - 1>();
@@ -531,7 +564,7 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
     }
     // ---- one group near the end of a segment, everything checked
     const int vt = cur.tv0 + lane;
-    process_group<BF16, false>(ws, g, st, vt, seg.v1, lt_mask, p.status);
+    process_group<BF16, false, TOPM>(ws, g, st, ts, vt, seg.v1, lt_mask, p.status);
     const bool last = cur.last_of_segment();
     cur.advance(p, s_off, esz);
     n = next_slot(n);
@@ -562,6 +595,14 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
       if (lane == 0 && slot_ok) {
         p.part_held[slot_id] = mine;
         p.part_stats[slot_id] = make_float4(st.c, S, U, __int_as_float(__popc(have)));
+        if (TOPM) {
+          TopmSegment rec;
+          rec.first = (int)(worker * ts.cap) + ts.first;
+          rec.n = ts.n > ts.cap ? -1 : ts.n - ts.first;
+          rec.floor = ts.floor;
+          rec.pad = 0;
+          p.topm_seg[slot_id] = rec;
+        }
       }
       __syncwarp();
       if (!cur.valid) break;
@@ -571,11 +612,11 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
   cp_async_wait<0>();
 }
 
-template <bool BF16>
+template <bool BF16, bool TOPM>
 __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_pass_kernel(PassParams p) {
   extern __shared__ __align__(16) unsigned char s_dyn[];
   chain_enter();
-  expand_pass_body<BF16>(p, s_dyn);
+  expand_pass_body<BF16, TOPM>(p, s_dyn);
 }
 
 // Expand and prune of a level in one launch, for small batches: the CTA that finishes last (an atomic ticket, nobody
@@ -587,7 +628,7 @@ __global__ void __launch_bounds__(kExpandThreads, kExpandCtasPerSm) expand_prune
   extern __shared__ __align__(16) unsigned char s_dyn[];
   __shared__ unsigned s_ticket;
   chain_enter();
-  expand_pass_body<BF16>(p, s_dyn);
+  expand_pass_body<BF16, false>(p, s_dyn);
   __threadfence();                                   // this CTA's records, before its ticket
   __syncthreads();
   if (threadIdx.x == 0) s_ticket = atomicAdd(t.ticket, 1u);
@@ -612,6 +653,12 @@ int expand_min_span(int vocab, int elem_bytes, int K) {
   return span < 256 ? 256 : span;
 }
 
+size_t topm_pool_vectors(size_t batch, size_t rows_per_seq, int vocab, int elem_bytes) {
+  const size_t vec = 16 / elem_bytes;
+  const size_t n = batch * rows_per_seq * ((vocab + vec - 1) / vec) / kTopmPoolDivisor + 4096;
+  return n < 0x7FFFFFFFu ? n : 0x7FFFFFFFu;          // records hold 32-bit positions
+}
+
 int max_splits_for(int vocab, int elem_bytes, int workers, int pad, int min_span) {
   const int vec = 16 / elem_bytes;
   const int vec_per_row = (vocab + vec - 1) / vec;
@@ -627,8 +674,10 @@ static size_t expand_dynamic_smem(int B) {
 cudaError_t prepare_expand_pass() {
   const int bytes = (int)expand_dynamic_smem(C2T_MAX_BATCH);
   const int fused = (int)expand_dynamic_smem(C2T_FUSED_MAX_BATCH);
-  cudaError_t e = cudaFuncSetAttribute(expand_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaError_t e = cudaFuncSetAttribute(expand_pass_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_pass_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_pass_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_pass_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_prune_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, fused);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(expand_prune_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, fused);
   return e;
@@ -646,8 +695,13 @@ cudaError_t launch_expand_prune(const PassParams &p, const TreeState &t, int lev
 
 cudaError_t launch_expand_pass(const PassParams &p, int dtype, int grid, cudaStream_t s) {
   const size_t smem = expand_dynamic_smem(p.B);
-  if (dtype == C2T_BF16) return launch_chained(expand_pass_kernel<true>, dim3(grid), dim3(kExpandThreads), smem, s, p);
-  return launch_chained(expand_pass_kernel<false>, dim3(grid), dim3(kExpandThreads), smem, s, p);
+  const bool bf16 = dtype == C2T_BF16;
+  if (p.topm_pool) {                                 // also sets the candidates of Eq. 3 aside
+    if (bf16) return launch_chained(expand_pass_kernel<true, true>, dim3(grid), dim3(kExpandThreads), smem, s, p);
+    return launch_chained(expand_pass_kernel<false, true>, dim3(grid), dim3(kExpandThreads), smem, s, p);
+  }
+  if (bf16) return launch_chained(expand_pass_kernel<true, false>, dim3(grid), dim3(kExpandThreads), smem, s, p);
+  return launch_chained(expand_pass_kernel<false, false>, dim3(grid), dim3(kExpandThreads), smem, s, p);
 }
 
 }  // namespace c2t

@@ -113,6 +113,8 @@ class Report:
     oracle_kept_nodes: list = field(default_factory=list)
     oracle_accept_len: list = field(default_factory=list)
     oracle_next_token: list = field(default_factory=list)
+    rows_expanded: int = 0               # active draft rows over all levels
+    rows_topm_from_pass: int = 0         # of those, rows whose Eq. 3 sums came from the vectors the pass set aside
 
     def line(self) -> str:
         return (f"seq={self.sequences} near_tie={self.near_tie_sequences} diverged={self.diverged_sequences} "
@@ -261,7 +263,13 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
         elif fused:
             ctx.c2t_expand_prune_level(l, draft_dev[l])
         else:
+            n_in = ctx.c2t_get_view()["frontier_n"].cpu().numpy().copy()
             ctx.c2t_expand_level(l, draft_dev[l])
+            from_pass = ctx.c2t_get_view()["topm_from_pass"]
+            if from_pass is not None:
+                fp = from_pass.cpu().numpy()
+                rep.rows_expanded += int(n_in.sum())
+                rep.rows_topm_from_pass += int(sum(fp[b, :n_in[b]].sum() for b in range(B)))
             ctx.c2t_prune(l)
         view = ctx.c2t_get_view()
         torch.cuda.synchronize()
@@ -310,7 +318,7 @@ def run_and_compare(ocfg, gcfg, draft_cpu, target_cpu, root, prefix, seqs=None, 
     ctx.c2t_build_verify()
     ctx.c2t_accept(target_dev)
     bits, per = ctx.c2t_status()
-    view = {k: v.cpu().numpy() for k, v in ctx.c2t_get_view().items()}
+    view = {k: v.cpu().numpy() for k, v in ctx.c2t_get_view().items() if v is not None}
     ver_g = {k: v.cpu().numpy() for k, v in ctx.verify.items()}
     acc_g = {k: v.cpu().numpy() for k, v in ctx.accepted.items()}
     # the walk that reads only the rows it visits must give the same answers

@@ -406,6 +406,22 @@ def test_truncated_entropy_top_m(dtype, V, M):
     case(4, V, 4, 8, 6, 24, 0.5, dtype, M=M)
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_truncated_entropy_comes_from_the_expand_pass(dtype):
+    """At the paper's vocabulary and M = 1000 the rows are read once: the pass sets the vectors aside that can hold
+    one of the M most probable tokens and Eq. 3's sums are taken from those (the view says for which rows)."""
+    rep = case(3, 128256, 3, 10, 8, 30, 0.0, dtype, M=1000, classifier="identity")
+    assert rep.rows_expanded == 3 * (1 + 8 + 8)
+    assert rep.rows_topm_from_pass >= 0.9 * rep.rows_expanded, (rep.rows_topm_from_pass, rep.rows_expanded)
+
+
+def test_truncated_entropy_rows_the_pass_cannot_serve_are_read_again():
+    """M close to V: fewer than M elements reach the floor above which the pass sets vectors aside, so every row
+    takes the second read (rows of equal values, where the regions run full, are among the special rows below)."""
+    rep = case(2, 6000, 2, 4, 4, 12, 0.0, torch.float32, M=4500, classifier="identity")
+    assert rep.rows_expanded == 2 * (1 + 4) and rep.rows_topm_from_pass == 0
+
+
 @pytest.mark.parametrize("kind", ["heavy_ties", "two_valued", "neg_inf", "uniform"])
 def test_truncated_entropy_on_special_rows(kind):
     """Many equal values around the M-th largest: equal values give equal terms, so only the count matters."""
@@ -419,6 +435,8 @@ def test_truncated_entropy_on_special_rows(kind):
     uniform = dict(allow_diverged=B, allow_kinds=("cross_row_tie",)) if kind == "uniform" else {}
     rep = run_and_compare(ocfg, gcfg, draft, target, root, prefix, **uniform)
     assert rep.status_bits == 0
+    if kind == "uniform":                # every vector reaches the floor: more than the pass has room for
+        assert rep.rows_topm_from_pass == 0
 
 
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
