@@ -447,6 +447,8 @@ def run_cuda(args) -> None:
     fp32_level = expand_full_level(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream, torch.float32, 4.0)
     # ... and on flat logits (temperature scale 1), where the kernel's work per element is at its largest
     scale1_level = expand_full_level(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream, torch.bfloat16, 1.0)
+    topm_level = expand_full_level(c2t, dev, (w1, b1, w2, b2), root, prefix, default_stream, torch.bfloat16, 4.0,
+                                   top_m=1000)
 
     # ---- the single-sequence configuration (latency-bound), timed per decode step; one GPU only
     single_seq = single_sequence_latency(c2t, dev, default_stream) if world == 1 else None
@@ -525,7 +527,8 @@ def run_cuda(args) -> None:
                      "fp32_logits_full_level": None if fp32_level is None else dict(
                          fp32_level, frac=fp32_level["gbs"] / peak),
                      "scale1_logits_full_level": None if scale1_level is None else dict(
-                         scale1_level, frac=scale1_level["gbs"] / peak, frac_of_8000=scale1_level["gbs"] / 8000.0)},
+                         scale1_level, frac=scale1_level["gbs"] / peak, frac_of_8000=scale1_level["gbs"] / 8000.0),
+                     "truncated_entropy_full_level": topm_level},
         "cpu_baseline": cpu_base,
     }
     print(json.dumps(line), flush=True)
@@ -554,21 +557,23 @@ def plant_accept_paths(ctx, target, V, depths=(2, 3, 4, 5)):
 
 
 def expand_full_level(c2t, dev, weights, root, prefix, stream, dtype=torch.float32, scale: float = 4.0,
-                      reps: int = 20):
+                      reps: int = 20, top_m: int = 0):
     """Times the expand kernel on full levels of the workload with other logits than the headline's: fp32 instead
     of bf16, or another temperature scale (levels 1-3, three distinct buffers, so every launch reads from DRAM).
-    Returns None if the frontier does not fill."""
+    top_m > 0: with the truncated entropy of Eq. 3, whose kernels run inside the same call (the time is then that of
+    the pass plus those).  Returns None if the frontier does not fill."""
     w = WORKLOAD
     B, V, K, F, N = w["B"], w["V"], w["K"], w["F"], w["N"]
     levels = 4
     w1, b1, w2, b2 = weights
     cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32 if dtype == torch.float32 else c2t.BF16, max_depth=levels,
                      topk=K, frontier_cap=F, budget=N, threshold=0.0, classifier=c2t.CLS_IDENTITY_JOINT,
-                     hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index)
+                     hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2, device=dev.index, entropy_top_m=top_m)
     ctx = c2t.Context(cfg)
     draft = [c2t_inputs.draft_logits(B, F, V, 0, l, dtype, scale, device=dev) for l in range(levels)]
     rows = []
     ms = []
+    from_pass = None
     for rep in range(reps + 3):
         ctx.c2t_begin_step(root, prefix, stream)
         for l in range(levels):
@@ -578,6 +583,8 @@ def expand_full_level(c2t, dev, weights, root, prefix, stream, dtype=torch.float
             a.record()
             ctx.c2t_expand_level(l, draft[l], stream)
             b.record()
+            if top_m and rep == 0 and l == 1:
+                from_pass = int(ctx.c2t_get_view()["topm_from_pass"].sum().item())
             ctx.c2t_prune(l, stream)
             if rep >= 3 and l >= 1:
                 ms.append((a, b))
@@ -588,9 +595,14 @@ def expand_full_level(c2t, dev, weights, root, prefix, stream, dtype=torch.float
     us = sum(t) / len(t)
     nbytes = B * F * V * (4 if dtype == torch.float32 else 2)
     ctx.close()
-    return {"rows": B * F, "bytes": nbytes, "us": us, "us_median": t[len(t) // 2], "us_min": t[0],
-            "gbs": nbytes / (us * 1e-6) / 1e9, "scale": scale, "dtype": "f32" if dtype == torch.float32 else "bf16",
-            "note": "threshold 0 with the identity classifier, so that every level has B*F active rows"}
+    out = {"rows": B * F, "bytes": nbytes, "us": us, "us_median": t[len(t) // 2], "us_min": t[0],
+           "gbs": nbytes / (us * 1e-6) / 1e9, "scale": scale, "dtype": "f32" if dtype == torch.float32 else "bf16",
+           "note": "threshold 0 with the identity classifier, so that every level has B*F active rows"}
+    if top_m:
+        out["entropy_top_m"] = top_m
+        out["rows_served_from_the_pass"] = from_pass
+        out["note"] += "; the time covers the pass, the per-row selection and the (empty) second-read launch"
+    return out
 
 
 def single_sequence_latency(c2t, dev, stream, steps: int = 60, sets: int = 4):
