@@ -1,20 +1,22 @@
 // Truncated entropy (Eq. 3): the sums over the M most probable tokens of every active draft row,
 // for configurations with entropy_top_m = M > 0.  The probabilities are those of the full softmax
-// (no renormalisation), so the expand pass still supplies the normaliser; this pass supplies
+// (no renormalisation), so the expand pass still supplies the normaliser; the kernels here supply
 //     S_M = sum over the top M of e^(x - m),   T_M = sum over the top M of e^(x - m) (x - m)
 // (m = the row maximum), from which  H_M = (ln Z * S_M - T_M) / Z.
 //
-// One CTA per active row.  The M-th largest value is found by a radix select on the order-
-// preserving 32-bit image of the values, one byte per step from the top (two steps for bf16,
-// whose images differ in the upper 16 bits only; four for fp32); then the terms above that
-// value are added, and as many copies of the term AT that value as are still missing (equal
-// values give equal terms, so which tokens are taken does not matter).
-//   Fast path: the row maximum is known from the expand pass, which runs just before; one sweep
-// copies the elements within two top key bytes of it to shared memory and everything else runs
-// on those.  General path (the guess failed): up to five sweeps over the row, which stays in L2;
-// the top byte is counted in registers from the maximum's bin downwards, the later bytes with a
-// 256-bin histogram in shared memory over the elements that still match.
-// An optional mode, not tuned further: about 2.4 times the expand pass on a 640-row level.
+// In both kernels the M-th largest value of a row is found on the order-preserving 32-bit image of
+// the values; then the terms above that value are added, and as many copies of the term AT that
+// value as are still missing (equal values give equal terms, so which tokens are taken does not
+// matter).
+//   topm_finish_kernel, one CTA per active row, works on the vectors that the expand pass set aside
+// (every vector with an element at or above a per-segment floor): if at least M elements reach the
+// highest floor among the row's segments, the M largest are among them.  The rows are not read again.
+//   topm_entropy_kernel, a persistent grid, takes the rows that kernel could not serve and reads them
+// once more.  Fast path: the row maximum is known from the expand pass; one sweep copies the elements
+// within two top key bytes of it to shared memory and the selection runs on those.  General path (that
+// guess failed too): a radix select over the row in up to five sweeps (the row stays in L2); the top
+// byte is counted in registers from the maximum's bin downwards, the later bytes with a 256-bin
+// histogram in shared memory over the elements that still match.
 #include "vocab_common.cuh"
 
 namespace c2t {
