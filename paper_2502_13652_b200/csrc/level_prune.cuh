@@ -252,11 +252,13 @@ template <int NW>
 struct PruneShared {
   double rowM[C2T_MAX_FRONTIER], rowL[C2T_MAX_FRONTIER], rowH[C2T_MAX_FRONTIER];
   double C[kMaxCand];
+  double logP[kMaxCand];                       // joint log-probability of every candidate
   unsigned long long keys[NW][kStageKeys];
   float w[5 * C2T_MAX_HIDDEN + 4];
   float x[kMaxCand];
   int tok[kMaxCand];
   double flogP[C2T_MAX_FRONTIER];              // joint log-probability of every frontier node
+  double fchat[C2T_MAX_FRONTIER];              // its smallest confidence on the path from the root
   int fnode[C2T_MAX_FRONTIER];                 // tree id of every frontier node
   int rowfault[C2T_MAX_FRONTIER];
   int scan[NW + 1];
@@ -303,13 +305,16 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
   int n = t.frontier_n[cur][b];
   const int row_off = t.row_off_draft[b];         // rows of earlier sequences in the expand pass
   const PassInfo info = *t.info_draft;            // (loads issued together with the one above)
-  // the frontier's nodes and their joint log-probabilities (Eq. 1's left factor), fetched now so that their two
-  // dependent loads run beside the rows' merges (slots past the frontier's size hold anything: kept in bounds, unused)
-  if (tid < F) {
-    int f = t.frontier_node[cur][(size_t)b * F + tid];
+  const int tree_base = t.tree_n[b];              // (needed last; its latency hides behind everything else)
+  // the frontier's nodes, their joint log-probabilities (Eq. 1's left factor) and path confidences: two dependent
+  // loads, issued by the last warp (the one least likely to have a row) so that they run beside the rows' merges;
+  // phases 2 and 4 read them, behind barriers (slots past the frontier's size hold anything: kept in bounds, unused)
+  if (warp == kTreeWarps - 1 && lane < F) {
+    int f = t.frontier_node[cur][(size_t)b * F + lane];
     f = f < 0 ? 0 : (f >= t.cap ? t.cap - 1 : f);
-    sh.fnode[tid] = f;
-    sh.flogP[tid] = t.tree_logP[(size_t)b * t.cap + f];
+    sh.fnode[lane] = f;
+    sh.flogP[lane] = t.tree_logP[(size_t)b * t.cap + f];
+    sh.fchat[lane] = t.tree_Chat[(size_t)b * t.cap + f];
   }
   n = n < 0 ? 0 : (n > F ? F : n);
   const size_t cbase = (size_t)b * F * K;
@@ -322,7 +327,7 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
     }
     return;
   }
-  __syncthreads();
+  // (no barrier here: phase 1 reads nothing that was written above)
 
   // ---- phase 1: one warp per row merges that row's partial records
   for (int j = warp; j < n; j += kTreeWarps) {
@@ -374,6 +379,7 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
     t.cand_token[cbase + c] = tok;
     t.cand_lp[cbase + c] = ok ? lp : NAN;
     t.cand_logP[cbase + c] = ok ? logP : NAN;
+    sh.logP[c] = logP;
     t.cand_H[cbase + c] = ok ? H : NAN;
     t.cand_C[cbase + c] = C;
   }
@@ -410,7 +416,7 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
   const int off_both = block_exclusive_scan<NT>(n_add | (n_sel << 16), s_scan, &tot_both);
   int off_add = off_both & 0xFFFF, off_sel = off_both >> 16;
   const int tot_add = tot_both & 0xFFFF, tot_sel = tot_both >> 16;
-  const int base = t.tree_n[b];
+  const int base = tree_base;
   const bool overflow = base + tot_add > t.cap;
   const size_t tb = (size_t)b * t.cap;
   for (int c = c0; c < c1; ++c) {
@@ -425,9 +431,9 @@ __device__ void prune_level_body(const TreeState &t, int level, const c2t_fronti
       t.tree_token[tb + id] = s_tok[c];
       t.tree_parent[tb + id] = f;
       t.tree_level[tb + id] = level + 1;
-      t.tree_logP[tb + id] = t.cand_logP[cbase + c];
+      t.tree_logP[tb + id] = sh.logP[c];              // (a node is only added if its candidate was in order)
       t.tree_C[tb + id] = s_C[c];
-      const double ch = t.tree_Chat[tb + f];
+      const double ch = sh.fchat[j];
       t.tree_Chat[tb + id] = s_C[c] < ch ? s_C[c] : ch;
     }
     if (s_sel[c] && !overflow) {
