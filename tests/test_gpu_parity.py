@@ -422,6 +422,14 @@ def test_truncated_entropy_rows_the_pass_cannot_serve_are_read_again():
     assert rep.rows_expanded == 2 * (1 + 4) and rep.rows_topm_from_pass == 0
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_truncated_entropy_with_both_routes_in_one_step(dtype):
+    """A small vocabulary with M = 64: some rows are served from the vectors the pass set aside, the others are
+    read again, within the same launches."""
+    rep = case(3, 1000, 3, 8, 6, 20, 0.0, dtype, M=64, classifier="identity")
+    assert 0 < rep.rows_topm_from_pass < rep.rows_expanded, (rep.rows_topm_from_pass, rep.rows_expanded)
+
+
 @pytest.mark.parametrize("kind", ["heavy_ties", "two_valued", "neg_inf", "uniform"])
 def test_truncated_entropy_on_special_rows(kind):
     """Many equal values around the M-th largest: equal values give equal terms, so only the count matters."""
