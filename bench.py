@@ -45,9 +45,9 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/expand_pass_kernel_bf16_B64_V128256.txt: the 64-row launch of level 0 and a 640-row launch.  The counters
 # belong to the kernel sources whose hash stands beside them: when a source changes the hash no longer matches and
 # the bench reports no traffic figure until the counters (and the hash) are taken again.
-EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 168.11e6}
+EXPAND_DRAM_BYTES = {"level0": 16.49e6, "full_level": 167.77e6}
 EXPAND_SOURCES = ("expand_pass.cu", "c2t_internal.h", "vocab_common.cuh")
-EXPAND_SOURCES_SHA16 = "0cd042730afd8295"
+EXPAND_SOURCES_SHA16 = "15c0e36ac9f6ade2"
 
 
 def expand_dram_bytes():
@@ -792,11 +792,13 @@ def run_profile(args) -> None:
     w = WORKLOAD
     B, V, D, K, F, N = w["B"], w["V"], w["D"], w["K"], w["F"], w["N"]
     w1, b1, w2, b2 = make_weights(w["hidden"])
-    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.BF16, max_depth=D, topk=K, frontier_cap=F, budget=N,
-                     threshold=w["beta"], hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2)
+    tdt = torch.float32 if args.profile_dtype == "f32" else torch.bfloat16
+    cfg = c2t.Config(batch=B, vocab=V, dtype=c2t.F32 if tdt == torch.float32 else c2t.BF16, max_depth=D, topk=K,
+                     frontier_cap=F, budget=N, threshold=w["beta"], hidden=w["hidden"], w1=w1, b1=b1, w2=w2, b2=b2,
+                     entropy_top_m=args.profile_top_m)
     ctx = c2t.Context(cfg)
-    draft = [c2t_inputs.draft_logits(B, F, V, 0, l, torch.bfloat16, device=dev) for l in range(2)]
-    target = c2t_inputs.target_logits(B, ctx.Nw, V, 0, torch.bfloat16, device=dev)
+    draft = [c2t_inputs.draft_logits(B, F, V, 0, l, tdt, device=dev) for l in range(2)]
+    target = c2t_inputs.target_logits(B, ctx.Nw, V, 0, tdt, device=dev)
     root = c2t_inputs.root_tokens(B, V, 0).to(dev)
     prefix = c2t_inputs.prefix_lengths(B).to(dev)
     for _ in range(args.warmup + args.steps):
@@ -821,6 +823,8 @@ def main() -> None:
     ap.add_argument("--profile", action="store_true",
                     help="small run for profiler captures: levels 0-1 of the workload plus rerank, verify "
                          "inputs and accept; no end-to-end leg, no CPU baseline")
+    ap.add_argument("--profile-dtype", choices=["bf16", "f32"], default="bf16", help="logits dtype of the --profile run")
+    ap.add_argument("--profile-top-m", type=int, default=0, help="entropy_top_m of the --profile run (Eq. 3)")
     args = ap.parse_args()
     if args.profile:
         args.steps = args.steps or 1

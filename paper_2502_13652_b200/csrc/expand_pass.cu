@@ -462,7 +462,13 @@ struct TopmState {
   uint4 *region;              // the warp's part of the pool
   int cap, n, first;          // its size in vectors; vectors set aside by the warp so far (may pass cap: then nothing more is stored); n when the segment began
   float floor;
+  unsigned long long keep;    // L2 policy of the stores: the vectors are read back right after the pass, the rows never again
 };
+
+__device__ __forceinline__ void store_keep_in_l2(uint4 *dst, const uint4 &q, unsigned long long policy) {
+  asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1, %2, %3, %4}, %5;"
+               ::"l"(dst), "r"(q.x), "r"(q.y), "r"(q.z), "r"(q.w), "l"(policy) : "memory");
+}
 
 // One group: vectors that meet the filter go to the queue, the others into the sums.  WHOLE:
 // no lane is past the segment's end (a vector past it holds the lowest value, below every floor).
@@ -479,7 +485,7 @@ __device__ __forceinline__ void process_group(WarpShared *ws, const Group &g, Se
       const bool c = vm[u] >= ts.floor;              // (false for a vector with a NaN; such a row is reported anyway)
       const unsigned cm = __ballot_sync(kFull, c);
       const int pos = ts.n + __popc(cm & lt_mask);
-      if (c && pos < ts.cap) ts.region[pos] = g.q[u];
+      if (c && pos < ts.cap) store_keep_in_l2(ts.region + pos, g.q[u], ts.keep);
       ts.n += __popc(cm);
     }
   }
@@ -584,8 +590,9 @@ __device__ __forceinline__ void expand_pass_body(const PassParams &p, unsigned c
   const unsigned lt_mask = (1u << lane) - 1u;
   SegState st;
   TopmState ts;
-  ts.region = nullptr; ts.cap = 0; ts.n = 0; ts.first = 0; ts.floor = INFINITY;
+  ts.region = nullptr; ts.cap = 0; ts.n = 0; ts.first = 0; ts.floor = INFINITY; ts.keep = 0ull;
   if (TOPM) {
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(ts.keep));
     const long long busy = div_floor(vtotal + span - 1, span);       // workers with a span of this launch
     const long long cap = div_floor(p.topm_pool_vecs, busy > 0 ? busy : 1);
     ts.cap = (int)(cap < 0x3FFFFFFF ? cap : 0x3FFFFFFF);
