@@ -546,7 +546,7 @@ struct TopmCollected {
   int32_t *done;
 };
 
-constexpr int kFinishThreads = 256;
+constexpr int kFinishThreads = 512;
 constexpr int kFinishCand = 8192;      // keys of a row that fit in shared memory (several CTAs per SM)
 constexpr int kFinishSegs = 64;        // segments of a row the kernel handles
 constexpr int kFinishBatch = 4;        // independent 16-byte loads a thread keeps in flight
