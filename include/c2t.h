@@ -138,7 +138,9 @@ int c2t_begin_step(c2t_ctx *ctx, const int32_t *root_tok_dev, const int32_t *pre
  * With cfg.entropy_top_m = M, 0 < M < V, the pass also sets aside the vectors that can hold one
  * of a row's M most probable tokens, and a second kernel takes the entropy over those M (Eq. 3),
  * which c2t_prune then uses instead, from them; only a row for which they do not suffice (see
- * c2t_view.topm_from_pass) is read once more.
+ * c2t_view.topm_from_pass) is read once more.  (Those M terms are added in fp64 in an order that
+ * depends on timing, so with M > 0 two runs may differ in the last bits of the entropy; everything
+ * else, and all of it with M = 0, repeats bit for bit.)
  *   logits_dev: [B, F, V] of cfg.dtype; element offset of (b, j, v) =
  *               b*seq_stride + j*row_stride + v.  Base address 16-byte aligned, both strides
  *               multiples of 16 bytes.  Rows of inactive slots are never read.
